@@ -1,0 +1,148 @@
+/*
+ * dmx.h — C ABI of the DYNAMIX data-parallel gradient step on one GPU.
+ *
+ * The operation (Algorithm 1, the inner "for each worker in parallel" body: each worker
+ * computes a gradient g_i at its own batch size x_i and the global model is updated under
+ * BSP; Section "State representation", paragraph "Training Statistical Efficiency Metrics":
+ * the controller reads gradient statistics, sigma_norm and sigma^2_norm):
+ *
+ *   K emulated workers hand in flat gradient vectors x_k[0..P) computed at batch sizes b_k.
+ *   One call forms the batch-size-weighted aggregate g = sum_k b_k x_k / sum_k b_k, the
+ *   statistics the batch-size policy reads, and the SGD-momentum update
+ *   m <- beta*m + g, theta <- theta - lr*m, prev_agg <- g.
+ *
+ * The paper states no formula for the aggregate, the statistics or the optimizer; the
+ * definitions below are this library's reading and are the contract.
+ *
+ * Conventions
+ *   - Every function returns DMX_OK (0) or a negative DMX_ERR_* code. Nothing throws,
+ *     aborts or traps, on the host or on the device.
+ *   - "HOST" / "DEVICE" on a pointer says which memory it addresses.
+ *   - dmx_step is asynchronous: it enqueues work on the given stream and returns. It does
+ *     not allocate, does not synchronise and copies nothing host-to-device (worker pointers,
+ *     weights and batch sizes travel as kernel arguments).
+ *   - A handle may be used from one stream at a time (its scratch is shared by its calls).
+ */
+#ifndef DMX_H_
+#define DMX_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dmx_handle dmx_handle;
+
+/* gradient element types */
+enum { DMX_F32 = 0, DMX_BF16 = 1 };
+
+/* return codes */
+enum {
+  DMX_OK = 0,
+  DMX_ERR_ARG = -1,      /* null pointer, K/P/S out of range, aliasing buffers, bad dtype  */
+  DMX_ERR_SEGMENTS = -2, /* segment table not o[0]=0 <= o[1] <= ... <= o[S]=P              */
+  DMX_ERR_BATCH = -3,    /* some batch size < 1                                            */
+  DMX_ERR_ALIGN = -4,    /* a device pointer is not 16-byte aligned                        */
+  DMX_ERR_NOMEM = -5,    /* host or device allocation failed                               */
+  DMX_ERR_CUDA = -6,     /* a CUDA runtime call failed (see dmx_last_cuda_error)           */
+  DMX_ERR_HANDLE = -7    /* handle is NULL, destroyed or corrupt                           */
+};
+
+/* limits */
+#define DMX_MAX_WORKERS 64
+#define DMX_MAX_SEGMENTS 65536
+#define DMX_MAX_PARAMS (((int64_t)1) << 40)
+
+/*
+ * Layout of out_state (fp32, length dmx_state_len = 16 + K + 2*S).
+ * With B = sum_k b_k, q_k = sum_j x_kj^2, A = sum_j g_j^2,
+ * D = sum_j sum_k b_k (x_kj - g_j)^2, a = prev_agg as passed in:
+ */
+enum {
+  DMX_ST_B_TOTAL = 0,      /* B                                                            */
+  DMX_ST_AGG_SQNORM = 1,   /* A                                                            */
+  DMX_ST_TR_SIGMA = 2,     /* tr(Sigma)^ = D/(K-1); unbiased for the per-sample covariance */
+                           /* trace when x_k is a mean of b_k i.i.d. samples; 0 if K == 1  */
+  DMX_ST_G2 = 3,           /* |G|^2^ = A - tr(Sigma)^/B; unbiased, may be <= 0             */
+  DMX_ST_GNS = 4,          /* gradient noise scale tr(Sigma)^ / |G|^2^ if |G|^2^ > 0 else 0
+                              (the quantity behind the paper's large->medium->small
+                              batch schedule, Section "RL Agent Inference Evaluation",
+                              paragraph "Batch Size Adaptation Dynamics")                      */
+  DMX_ST_COS_PREV = 5,     /* <g,a> / sqrt(A * |a|^2) if both norms > 0 else 0             */
+  DMX_ST_DOT_PREV = 6,     /* <g,a>                                                        */
+  DMX_ST_PREV_SQNORM = 7,  /* |a|^2                                                        */
+  DMX_ST_SIGMA2_NORM = 8,  /* sigma^2_norm = tr(Sigma)^ / (B*A) if A > 0 else 0            */
+  DMX_ST_SIGMA_NORM = 9,   /* sigma_norm = sqrt(max(sigma^2_norm, 0))                      */
+  DMX_ST_WMEAN_SQNORM = 10,/* sum_k b_k q_k / B                                            */
+  DMX_ST_FLAGS = 11,       /* bit mask stored as a float, DMX_FLAG_*                       */
+  DMX_ST_HDR = 16          /* 12..15 reserved (0); then q_k [K], V_s [S], N_s [S]          */
+};
+/* V_s = (sum_{j in s} sum_k b_k (x_kj-g_j)^2)/(K-1): segment s's additive share of
+ * tr(Sigma)^ (0 if K == 1).  N_s = sum_{j in s} g_j^2.  Empty segments give 0. */
+
+enum {
+  DMX_FLAG_NONFINITE = 1,  /* some q_k, |a|^2 or A is not finite as fp32                   */
+  DMX_FLAG_G2_NONPOS = 2,  /* |G|^2^ <= 0 (or NaN): gns reported as 0                      */
+  DMX_FLAG_COS_UNDEF = 4,  /* A == 0 or |a|^2 == 0 (first step): cosine reported as 0      */
+  DMX_FLAG_SINGLE = 8,     /* K == 1: no across-worker variance                            */
+  DMX_FLAG_INTERNAL = 16   /* a bounded wait inside the kernel ran out; results invalid    */
+};
+
+/*
+ * dmx_create — validate (K, P, segment table), choose the launch configuration for the
+ * current CUDA device, build the device-side tables and allocate the reduction scratch.
+ *   K            number of workers, 1..DMX_MAX_WORKERS
+ *   P            number of parameters, 1..DMX_MAX_PARAMS-1
+ *   seg_offsets  HOST, S+1 entries: o[0]=0 <= o[1] <= ... <= o[S]=P; segment s is
+ *                [o[s], o[s+1]); zero-length segments allowed; the table is copied
+ *   S            number of segments, 1..DMX_MAX_SEGMENTS
+ *   grad_dtype   DMX_F32 or DMX_BF16 (params, momentum, prev_agg, out_state are fp32)
+ *   out          HOST, receives the handle
+ * Errors: DMX_ERR_ARG, DMX_ERR_SEGMENTS, DMX_ERR_NOMEM, DMX_ERR_CUDA. Synchronous.
+ */
+int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dtype,
+               dmx_handle** out);
+
+/* 16 + K + 2*S, or DMX_ERR_HANDLE. */
+int dmx_state_len(const dmx_handle* h);
+
+/*
+ * dmx_step — one iteration: aggregate, statistics, SGD-momentum update, state vector.
+ *   grad_ptrs    HOST array of K DEVICE pointers; each addresses P elements of grad_dtype,
+ *                16-byte aligned, read only
+ *   batch_sizes  HOST array of K ints, each >= 1
+ *   params       DEVICE, P fp32, 16-byte aligned, updated in place: theta - lr*m'
+ *   momentum     DEVICE, P fp32, 16-byte aligned, updated in place: m' = beta*m + g
+ *   lr, beta     learning rate and momentum coefficient (used as fp32)
+ *   prev_agg     DEVICE, P fp32, 16-byte aligned; in: the previous step's aggregate
+ *                (zeros before the first step); out: this step's aggregate g
+ *   out_state    DEVICE, dmx_state_len(h) fp32, 4-byte aligned, fully overwritten
+ *   cuda_stream  a cudaStream_t passed as void*; NULL = the legacy default stream
+ * Buffers stay owned by the caller and must stay alive and untouched until the stream has
+ * passed the step. params, momentum, prev_agg, out_state and the gradient buffers must be
+ * pairwise disjoint (checked by address range; gradient buffers may alias one another).
+ * Argument errors return before anything is enqueued: DMX_ERR_HANDLE, DMX_ERR_ARG,
+ * DMX_ERR_BATCH, DMX_ERR_ALIGN; a failed launch returns DMX_ERR_CUDA.
+ * Data problems (non-finite inputs, zero norms, |G|^2^ <= 0) are not errors: they set
+ * bits in out_state[DMX_ST_FLAGS].
+ */
+int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes,
+             float* params, float* momentum, float lr, float beta, float* prev_agg,
+             float* out_state, void* cuda_stream);
+
+/* Frees the tables and the scratch. NULL is accepted. The caller makes sure no step of
+ * this handle is still running. */
+int dmx_destroy(dmx_handle* h);
+
+/* Static, NUL-terminated description of a return code. */
+const char* dmx_strerror(int code);
+
+/* The cudaError_t (as int) of the last failed CUDA call made by this library on the
+ * calling thread, 0 if none. */
+int dmx_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DMX_H_ */

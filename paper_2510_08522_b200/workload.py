@@ -1,0 +1,252 @@
+"""Seeded synthetic workloads: the only module the CUDA path's tests and the oracle's tests share.
+
+It holds no arithmetic of the gradient step itself: only a counter-based random generator
+(Philox4x32-10, from its published definition: Salmon, Moraes, Dror, Shaw, "Parallel random
+numbers: as easy as 1, 2, 3", SC'11), the recipes that turn it into gradients, segment tables
+and batch-size schedules, and the bf16 storage conversions.
+
+The five workloads stand in for the gradient traffic of the models the paper trains (VGG and
+ResNet variants on CIFAR, Section "Workloads and Datasets") and for a BERT-large sized model,
+by size and structure only: no dataset, weights or real gradients are involved.
+
+    mu_j            ~ N(0, 0.01)                  common signal (variance 0.01, std 0.1)
+    x_kj            = round_dtype(mu_j + sigma_k * z_kj / sqrt(b_k)),  z ~ N(0,1) i.i.d.
+    mu              <- mu + N(0, 1e-3) per element per step (workloads with drift)
+    theta_0         ~ N(0, 0.05^2),  m_0 = 0,  prev_agg_0 = 0
+
+Random numbers are addressed, not drawn in sequence: the four normals of elements 4i..4i+3 of
+stream (tag, c2, c3) come from Philox counter (i lo, i hi, c2, c3) under key (seed, tag), so
+any slice regenerates on its own and the GPU fill kernels and this host twin agree on the
+integers (the float transforms agree to rounding).
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+
+import numpy as np
+
+F32, BF16 = 0, 1
+
+TAG_MU, TAG_DRIFT, TAG_NOISE, TAG_THETA, TAG_HOST = 1, 2, 3, 4, 5
+
+MU_STD = 0.1                    # sqrt(0.01)
+DRIFT_STD = math.sqrt(1e-3)
+THETA_STD = 0.05
+
+_M0, _M1 = 0xD2511F53, 0xCD9E8D57
+_W0, _W1 = 0x9E3779B9, 0xBB67AE85
+_MASK = 0xFFFFFFFF
+
+
+def philox4x32(c0, c1, c2, c3, k0, k1):
+    """Philox4x32-10 on numpy uint64 arrays holding 32-bit words; returns four such arrays."""
+    c0 = np.asarray(c0, dtype=np.uint64); c1 = np.asarray(c1, dtype=np.uint64)
+    c2 = np.asarray(c2, dtype=np.uint64); c3 = np.asarray(c3, dtype=np.uint64)
+    c0, c1, c2, c3 = np.broadcast_arrays(c0, c1, c2, c3)
+    k0 = int(k0) & _MASK
+    k1 = int(k1) & _MASK
+    m = np.uint64(_MASK)
+    sh = np.uint64(32)
+    for _ in range(10):
+        p0 = np.uint64(_M0) * c0
+        p1 = np.uint64(_M1) * c2
+        hi0, lo0 = p0 >> sh, p0 & m
+        hi1, lo1 = p1 >> sh, p1 & m
+        c0, c1, c2, c3 = (hi1 ^ c1 ^ np.uint64(k0)), lo1, (hi0 ^ c3 ^ np.uint64(k1)), lo0
+        k0 = (k0 + _W0) & _MASK
+        k1 = (k1 + _W1) & _MASK
+    return c0, c1, c2, c3
+
+
+def normals(seed, tag, c2, c3, j0, n):
+    """Standard normals (float64) of elements [j0, j0+n) of stream (tag, c2, c3)."""
+    i0, i1 = j0 // 4, (j0 + n + 3) // 4
+    idx = np.arange(i0, i1, dtype=np.uint64)
+    r = philox4x32(idx & np.uint64(_MASK), idx >> np.uint64(32), c2, c3, seed, tag)
+    u = [(x.astype(np.float64) + 0.5) * 2.0 ** -32 for x in r]
+    rad0 = np.sqrt(-2.0 * np.log(u[0]))
+    rad1 = np.sqrt(-2.0 * np.log(u[2]))
+    z = np.empty((i1 - i0, 4), dtype=np.float64)
+    z[:, 0] = rad0 * np.cos(2.0 * np.pi * u[1])
+    z[:, 1] = rad0 * np.sin(2.0 * np.pi * u[1])
+    z[:, 2] = rad1 * np.cos(2.0 * np.pi * u[3])
+    z[:, 3] = rad1 * np.sin(2.0 * np.pi * u[3])
+    z = z.reshape(-1)
+    return z[j0 - 4 * i0: j0 - 4 * i0 + n]
+
+
+def host_words(seed, purpose, n, c3=0):
+    """n uint32 words for host-side draws (tables, batch sizes), word i of (purpose, c3)."""
+    idx = np.arange((n + 3) // 4, dtype=np.uint64)
+    r = philox4x32(idx, 0, purpose, c3, seed, TAG_HOST)
+    return np.stack(r, axis=1).reshape(-1)[:n].astype(np.uint64)
+
+
+def f32_to_bf16_bits(x):
+    """fp32 -> bf16 bit patterns (uint16), round to nearest even; finite inputs."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    return ((u + np.uint64(0x7FFF) + ((u >> np.uint64(16)) & np.uint64(1))) >> np.uint64(16)).astype(np.uint16)
+
+
+def bf16_bits_to_f32(b):
+    return (np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+# ---------------------------------------------------------------------------------------------
+# segment tables
+
+
+def equal_segments(P, S):
+    return np.array([P * s // S for s in range(S + 1)], dtype=np.int64)
+
+
+def _lognormal_sizes(total, n, seed, purpose):
+    """n sizes >= 1 summing to `total`, proportional to exp(1.5 * N(0,1)); the remainder goes
+    to the largest. Sizes are not rounded to any multiple, so boundaries fall at every
+    residue mod 4 and mod 8, like a real layer table with its bias and norm vectors."""
+    z = normals(seed, TAG_HOST, purpose, 1, 0, n)
+    ell = np.exp(1.5 * z)
+    sizes = np.maximum(1, np.floor(total * ell / ell.sum())).astype(np.int64)
+    sizes[np.argmax(sizes)] += total - sizes.sum()
+    assert sizes.min() >= 1 and sizes.sum() == total
+    return sizes
+
+
+def lognormal_segments(P, S, seed):
+    return np.concatenate([[0], np.cumsum(_lognormal_sizes(P, S, seed, 10))]).astype(np.int64)
+
+
+def two_heavy_segments(P, S, seed, heavy=((26, 0.65), (28, 0.15))):
+    """S segments; the listed ones hold the given fractions of P (together 80 %), the others
+    share the rest log-normally (a VGG-like table: two huge dense layers)."""
+    sizes = np.zeros(S, dtype=np.int64)
+    taken = 0
+    for idx, frac in heavy:
+        sizes[idx] = int(P * frac)
+        taken += sizes[idx]
+    rest = [s for s in range(S) if s not in dict(heavy)]
+    sizes[rest] = _lognormal_sizes(P - taken, len(rest), seed, 11)
+    return np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+
+
+# ---------------------------------------------------------------------------------------------
+# workloads
+
+
+@dataclasses.dataclass(frozen=True)
+class Workload:
+    name: str
+    K: int
+    P: int
+    S: int
+    dtype: int
+    steps: int
+    seed: int
+    segments: str           # "equal" | "lognormal" | "two_heavy"
+    batches: str            # "fixed4" | "once32" | "redraw16" | "tiers" | "walk32"
+    drift: bool
+    sigma_spread: bool = False
+    lr: float = 0.1
+    beta: float = 0.9
+
+    @property
+    def elem_bytes(self):
+        return 4 if self.dtype == F32 else 2
+
+    @property
+    def bytes_per_step(self):
+        """Algorithmic HBM bytes of one step: every gradient element read once; params,
+        momentum and prev_agg each read once and written once."""
+        return self.P * (self.K * self.elem_bytes + 24)
+
+    def scaled(self, P, steps=None, S=None):
+        """Same structure at another size (parity tests at sizes the oracle finishes fast)."""
+        return dataclasses.replace(self, name="%s@P=%d" % (self.name, P), P=int(P),
+                                   steps=self.steps if steps is None else steps,
+                                   S=self.S if S is None else S)
+
+    def segment_table(self):
+        if self.segments == "equal":
+            return equal_segments(self.P, self.S)
+        if self.segments == "lognormal":
+            return lognormal_segments(self.P, self.S, self.seed)
+        if self.segments == "two_heavy":
+            return two_heavy_segments(self.P, self.S, self.seed)
+        raise ValueError(self.segments)
+
+    def sigma(self):
+        """Per-worker noise scale sigma_k (1 unless the workload spreads it over U(0.5, 2))."""
+        if not self.sigma_spread:
+            return np.ones(self.K, dtype=np.float64)
+        w = host_words(self.seed, 20, self.K).astype(np.float64)
+        return 0.5 + 1.5 * (w + 0.5) * 2.0 ** -32
+
+    def batch_sizes(self, step):
+        K = self.K
+        if self.batches == "fixed4":
+            base = np.array([32, 64, 96, 128], dtype=np.int64)
+            return np.resize(base, K).astype(np.int32)
+        if self.batches == "once32":          # uniform over {32, 64, ..., 256}, drawn once
+            return (32 * (1 + host_words(self.seed, 21, K) % 8)).astype(np.int32)
+        if self.batches == "redraw16":        # multiples of 16 in [16, 512], redrawn every 10 steps
+            return (16 * (1 + host_words(self.seed, 22, K, c3=step // 10) % 32)).astype(np.int32)
+        if self.batches == "tiers":           # four tiers, K/4 workers each
+            tiers = np.array([32, 64, 128, 256], dtype=np.int64)
+            return tiers[(np.arange(K) * 4) // K].astype(np.int32)
+        if self.batches == "walk32":          # +-32 every step within [16, 1024]
+            b = (32 * (1 + host_words(self.seed, 23, K) % 32)).astype(np.int64)
+            for t in range(1, step + 1):
+                coin = host_words(self.seed, 24, K, c3=t) & np.uint64(1)
+                b = np.clip(b + np.where(coin == 1, 32, -32), 16, 1024)
+            return b.astype(np.int32)
+        raise ValueError(self.batches)
+
+    def grad_scale(self, step):
+        """scale_k = sigma_k / sqrt(b_k), as the fp32 values the fill kernels receive."""
+        return (self.sigma() / np.sqrt(self.batch_sizes(step).astype(np.float64))).astype(np.float32)
+
+
+WORKLOADS = [
+    Workload("cfg0-K4-1M-f32", 4, 1_048_576, 4, F32, 1, 0, "equal", "fixed4", False),
+    Workload("cfg1-K8-resnet18-f32", 8, 11_689_512, 62, F32, 100, 1, "lognormal", "once32", True),
+    Workload("cfg2-K16-resnet50-bf16", 16, 25_557_032, 161, BF16, 200, 2, "lognormal", "redraw16", True),
+    Workload("cfg3-K32-vgg16-f32", 32, 138_357_544, 32, F32, 50, 3, "two_heavy", "tiers", True),
+    Workload("cfg4-K32-bertlarge-bf16", 32, 340_000_000, 390, BF16, 50, 4, "lognormal", "walk32", True,
+             sigma_spread=True),
+]
+
+
+# ---------------------------------------------------------------------------------------------
+# host twin of the fill kernels (small sizes; float transforms agree with the GPU to rounding)
+
+
+class HostProblem:
+    """A workload materialised in numpy, one step at a time. Arrays are what `dmx_step`
+    and the oracle consume: float32 (or bf16 bit patterns as uint16) gradients, float32 state."""
+
+    def __init__(self, wl: Workload):
+        self.wl = wl
+        self.seg = wl.segment_table()
+        P = wl.P
+        self.mu = (MU_STD * normals(wl.seed, TAG_MU, 0, 0, 0, P)).astype(np.float32)
+        self.params0 = (THETA_STD * normals(wl.seed, TAG_THETA, 0, 0, 0, P)).astype(np.float32)
+        self.step_index = 0
+
+    def grads(self):
+        """Gradients of the current step (list of K arrays) and its batch sizes."""
+        wl, t = self.wl, self.step_index
+        b = wl.batch_sizes(t)
+        scale = wl.grad_scale(t)
+        out = []
+        for k in range(wl.K):
+            z = normals(wl.seed, TAG_NOISE, k, t, 0, wl.P).astype(np.float32)
+            x = (self.mu + scale[k] * z).astype(np.float32)
+            out.append(f32_to_bf16_bits(x) if wl.dtype == BF16 else x)
+        return out, b
+
+    def advance(self):
+        self.step_index += 1
+        if self.wl.drift:
+            d = (DRIFT_STD * normals(self.wl.seed, TAG_DRIFT, 0, self.step_index, 0, self.wl.P))
+            self.mu = (self.mu + d.astype(np.float32)).astype(np.float32)
