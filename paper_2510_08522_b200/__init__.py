@@ -1,0 +1,7 @@
+"""B200-native gradient step for batch-size-controlled data-parallel training (DYNAMIX hot path).
+
+`binding` mirrors the C ABI of include/dmx.h; `workload` holds the seeded synthetic inputs;
+`build` compiles the CUDA sources in-tree.
+"""
+from .binding import (BF16, F32, Dmx, DmxError, dmx_create, dmx_destroy, dmx_last_cuda_error,  # noqa: F401
+                      dmx_state_len, dmx_step, strerror)

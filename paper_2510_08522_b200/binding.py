@@ -1,0 +1,132 @@
+"""Thin ctypes binding of the C ABI in include/dmx.h: same names, argument marshalling only.
+
+Every step of the path runs in the CUDA library. There is no CPU fallback: if the shared
+object is missing or fails to load, importing callers get an error.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+from . import build as _build
+
+F32, BF16 = 0, 1
+OK = 0
+ERR_ARG, ERR_SEGMENTS, ERR_BATCH, ERR_ALIGN, ERR_NOMEM, ERR_CUDA, ERR_HANDLE = -1, -2, -3, -4, -5, -6, -7
+ST_B_TOTAL, ST_AGG_SQNORM, ST_TR_SIGMA, ST_G2, ST_GNS, ST_COS_PREV, ST_DOT_PREV, ST_PREV_SQNORM = range(8)
+ST_SIGMA2_NORM, ST_SIGMA_NORM, ST_WMEAN_SQNORM, ST_FLAGS = 8, 9, 10, 11
+ST_HDR = 16
+FLAG_NONFINITE, FLAG_G2_NONPOS, FLAG_COS_UNDEF, FLAG_SINGLE, FLAG_INTERNAL = 1, 2, 4, 8, 16
+
+EXPORTS = ("dmx_create", "dmx_state_len", "dmx_step", "dmx_destroy", "dmx_strerror", "dmx_last_cuda_error")
+
+_lib = None
+
+
+class DmxError(RuntimeError):
+    def __init__(self, code, where=""):
+        self.code = code
+        super().__init__("%s: %s (%d)" % (where or "dmx", strerror(code), code))
+
+
+def lib():
+    """Load lib/libdmx.so (built in-tree by `python -m paper_2510_08522_b200.build`)."""
+    global _lib
+    if _lib is None:
+        path = _build.lib_path("libdmx.so")
+        if not os.path.exists(path):
+            raise RuntimeError("CUDA library %s is not built; run `python -m paper_2510_08522_b200.build`" % path)
+        L = ctypes.CDLL(path)
+        vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float
+        L.dmx_create.argtypes = [i32, i64, vp, i32, i32, ctypes.POINTER(vp)]
+        L.dmx_create.restype = i32
+        L.dmx_state_len.argtypes = [vp]
+        L.dmx_state_len.restype = i32
+        L.dmx_step.argtypes = [vp, vp, vp, vp, vp, f32, f32, vp, vp, vp]
+        L.dmx_step.restype = i32
+        L.dmx_destroy.argtypes = [vp]
+        L.dmx_destroy.restype = i32
+        L.dmx_strerror.argtypes = [i32]
+        L.dmx_strerror.restype = ctypes.c_char_p
+        L.dmx_last_cuda_error.argtypes = []
+        L.dmx_last_cuda_error.restype = i32
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().dmx_strerror(int(code)).decode()
+
+
+def dmx_create(K, P, seg_offsets, grad_dtype=F32):
+    """-> (code, handle). seg_offsets: sequence of S+1 ints (host)."""
+    seg = (ctypes.c_int64 * len(seg_offsets))(*[int(v) for v in seg_offsets])
+    h = ctypes.c_void_p()
+    rc = lib().dmx_create(int(K), int(P), seg, len(seg_offsets) - 1, int(grad_dtype), ctypes.byref(h))
+    return rc, h
+
+
+def dmx_state_len(h) -> int:
+    return lib().dmx_state_len(h)
+
+
+def dmx_step(h, grad_ptrs, batch_sizes, params, momentum, lr, beta, prev_agg, out_state, stream=0) -> int:
+    """All buffer arguments are raw device addresses (ints); grad_ptrs / batch_sizes are
+    host sequences of length K."""
+    K = len(grad_ptrs)
+    gp = (ctypes.c_void_p * K)(*[int(p) for p in grad_ptrs])
+    bs = (ctypes.c_int32 * K)(*[int(b) for b in batch_sizes])
+    return lib().dmx_step(h, gp, bs, int(params), int(momentum), float(lr), float(beta), int(prev_agg),
+                          int(out_state), int(stream) if stream else None)
+
+
+def dmx_destroy(h) -> int:
+    return lib().dmx_destroy(h)
+
+
+def dmx_last_cuda_error() -> int:
+    return lib().dmx_last_cuda_error()
+
+
+class Dmx:
+    """Convenience owner of a handle for torch callers: tensors in, raw pointers through the C ABI."""
+
+    def __init__(self, K, P, seg_offsets, grad_dtype=F32):
+        import torch
+        self._torch = torch
+        self.K, self.P, self.S, self.dtype = int(K), int(P), len(seg_offsets) - 1, int(grad_dtype)
+        rc, self._h = dmx_create(K, P, seg_offsets, grad_dtype)
+        if rc != OK:
+            self._h = None
+            raise DmxError(rc, "dmx_create")
+        self.state_len = dmx_state_len(self._h)
+
+    def step(self, grads, batch_sizes, params, momentum, lr, beta, prev_agg, out_state=None, stream=None):
+        torch = self._torch
+        want = torch.float32 if self.dtype == F32 else torch.bfloat16
+        if len(grads) != self.K or len(batch_sizes) != self.K:
+            raise DmxError(ERR_ARG, "dmx_step")
+        for g in grads:
+            if g.dtype != want or not g.is_cuda or not g.is_contiguous() or g.numel() != self.P:
+                raise DmxError(ERR_ARG, "dmx_step (gradient tensor)")
+        for t in (params, momentum, prev_agg):
+            if t.dtype != torch.float32 or not t.is_cuda or not t.is_contiguous() or t.numel() != self.P:
+                raise DmxError(ERR_ARG, "dmx_step (state tensor)")
+        if out_state is None:
+            out_state = torch.empty(self.state_len, dtype=torch.float32, device=params.device)
+        elif out_state.dtype != torch.float32 or out_state.numel() != self.state_len or not out_state.is_cuda:
+            raise DmxError(ERR_ARG, "dmx_step (out_state)")
+        if stream is None:
+            stream = torch.cuda.current_stream(params.device).cuda_stream
+        rc = dmx_step(self._h, [g.data_ptr() for g in grads], batch_sizes, params.data_ptr(), momentum.data_ptr(),
+                      lr, beta, prev_agg.data_ptr(), out_state.data_ptr(), stream)
+        if rc != OK:
+            raise DmxError(rc, "dmx_step")
+        return out_state
+
+    def close(self):
+        if getattr(self, "_h", None):
+            dmx_destroy(self._h)
+            self._h = None
+
+    __del__ = close

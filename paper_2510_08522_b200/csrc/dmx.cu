@@ -1,0 +1,330 @@
+// dmx.cu — host side of the C ABI declared in dmx.h: validation, launch planning, the two
+// launches of a step (fused pass, finalize). All device work of a step is in dmx_kernels.cuh.
+#include "dmx.h"
+
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "dmx_kernels.cuh"
+
+namespace {
+
+thread_local int g_last_cuda = 0;
+
+bool cuda_ok(cudaError_t e) {
+  if (e == cudaSuccess) return true;
+  g_last_cuda = (int)e;
+  (void)cudaGetLastError();
+  return false;
+}
+
+constexpr uint64_t kMagic = 0x444d585f48414e44ull;  // "DMX_HAND"
+
+typedef void (*StepKernel)(const dmx::StepArgs);
+
+struct Plan {
+  StepKernel kernel = nullptr;
+  int threads = 0;       // threads per CTA
+  int tile = 0;          // elements per tile
+  size_t smem = 0;       // dynamic shared memory
+  int grid = 0;
+};
+
+int env_int(const char* name, int dflt) {
+  const char* v = std::getenv(name);
+  if (!v || !*v) return dflt;
+  return std::atoi(v);
+}
+
+template <typename T>
+bool upload(const std::vector<T>& v, T** dptr) {
+  *dptr = nullptr;
+  if (v.empty()) return true;
+  if (!cuda_ok(cudaMalloc((void**)dptr, v.size() * sizeof(T)))) return false;
+  return cuda_ok(cudaMemcpy(*dptr, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice));
+}
+
+}  // namespace
+
+struct dmx_handle {
+  uint64_t magic = kMagic;
+  int K = 0, S = 0, dtype = 0, device = 0;
+  int64_t P = 0;
+  Plan plan;
+  int nchunks = 0, nslots = 0;
+  // device tables
+  int64_t* seg_off = nullptr;
+  int32_t *cta_chunk0 = nullptr, *chunk_tile0 = nullptr, *chunk_seg0 = nullptr, *chunk_slot0 = nullptr;
+  int32_t *seg_chunk_lo = nullptr, *seg_chunk_hi = nullptr;
+  // device scratch
+  float *rows = nullptr, *slots = nullptr;
+  double* colsum = nullptr;
+  unsigned* flags = nullptr;  // [0] ticket, [1] err
+};
+
+namespace {
+
+// Kernel table: capacity KT in {4, 8, 16, 32, 64} (runtime K <= KT), fp32 / bf16 gradients.
+template <int KT, bool BF16>
+Plan direct_plan() {
+  constexpr int NW = 8;
+  constexpr int U = BF16 ? 4 : 8;
+  Plan p;
+  p.kernel = dmx::direct_kernel<KT, BF16, NW, U>;
+  p.threads = NW * 32;
+  p.tile = NW * 32 * dmx::Elem<BF16>::VEC;
+  p.smem = 0;
+  return p;
+}
+
+template <bool BF16>
+Plan pick_direct(int K) {
+  if (K <= 4) return direct_plan<4, BF16>();
+  if (K <= 8) return direct_plan<8, BF16>();
+  if (K <= 16) return direct_plan<16, BF16>();
+  if (K <= 32) return direct_plan<32, BF16>();
+  return direct_plan<64, BF16>();
+}
+
+// Pipelined (bulk-copy ring) kernels. Ring geometry: 8 consumer warps, 4 gradient streams per
+// stage; as many stages as fit beside the double-buffered state stage.
+template <int KT, bool BF16>
+Plan pipe_plan() {
+  typedef dmx::PipeCfg<KT, BF16, 8, 4, BF16 ? 10 : 12, 2> C;
+  Plan p;
+  p.kernel = dmx::pipe_kernel<C>;
+  p.threads = C::THREADS;
+  p.tile = C::T;
+  p.smem = C::SMEM;
+  return p;
+}
+
+template <bool BF16>
+Plan pick_pipe(int K) {
+  if (K <= 4) return pipe_plan<4, BF16>();
+  if (K <= 8) return pipe_plan<8, BF16>();
+  if (K <= 16) return pipe_plan<16, BF16>();
+  if (K <= 32) return pipe_plan<32, BF16>();
+  return pipe_plan<64, BF16>();
+}
+
+void free_handle(dmx_handle* h) {
+  if (!h) return;
+  cudaFree(h->seg_off); cudaFree(h->cta_chunk0); cudaFree(h->chunk_tile0); cudaFree(h->chunk_seg0);
+  cudaFree(h->chunk_slot0); cudaFree(h->seg_chunk_lo); cudaFree(h->seg_chunk_hi);
+  cudaFree(h->rows); cudaFree(h->slots); cudaFree(h->colsum); cudaFree(h->flags);
+  (void)cudaGetLastError();
+  h->magic = 0;
+  delete h;
+}
+
+// Segment holding element j: the unique s with o[s] <= j < o[s+1].
+int segment_of(const int64_t* o, int S, int64_t j) {
+  return (int)(std::upper_bound(o, o + S + 1, j) - o) - 1;
+}
+
+bool overlap(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
+  return x < y + nb && y < x + na;
+}
+
+}  // namespace
+
+extern "C" {
+
+int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dtype, dmx_handle** out) {
+  if (!out) return DMX_ERR_ARG;
+  *out = nullptr;
+  if (K < 1 || K > DMX_MAX_WORKERS || P < 1 || P >= DMX_MAX_PARAMS || S < 1 || S > DMX_MAX_SEGMENTS ||
+      !seg_offsets || (grad_dtype != DMX_F32 && grad_dtype != DMX_BF16))
+    return DMX_ERR_ARG;
+  if (seg_offsets[0] != 0 || seg_offsets[S] != P) return DMX_ERR_SEGMENTS;
+  for (int s = 0; s < S; ++s)
+    if (seg_offsets[s] > seg_offsets[s + 1]) return DMX_ERR_SEGMENTS;
+
+  dmx_handle* h = new (std::nothrow) dmx_handle;
+  if (!h) return DMX_ERR_NOMEM;
+  h->K = K; h->P = P; h->S = S; h->dtype = grad_dtype;
+  cudaDeviceProp prop;
+  if (!cuda_ok(cudaGetDevice(&h->device)) || !cuda_ok(cudaGetDeviceProperties(&prop, h->device))) {
+    free_handle(h);
+    return DMX_ERR_CUDA;
+  }
+
+  // DMX_KERNEL=direct selects the plain-load kernel (a tuning and cross-check knob); the
+  // default is the bulk-copy pipeline.
+  const char* kv = std::getenv("DMX_KERNEL");
+  const bool direct = kv && std::strcmp(kv, "direct") == 0;
+  Plan plan = direct ? (grad_dtype == DMX_BF16 ? pick_direct<true>(K) : pick_direct<false>(K))
+                     : (grad_dtype == DMX_BF16 ? pick_pipe<true>(K) : pick_pipe<false>(K));
+  if (plan.smem > 48 * 1024 &&
+      !cuda_ok(cudaFuncSetAttribute(plan.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem))) {
+    free_handle(h);
+    return DMX_ERR_CUDA;
+  }
+  int occ = 0;
+  if (!cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, plan.kernel, plan.threads, plan.smem)) || occ < 1) {
+    free_handle(h);
+    return DMX_ERR_CUDA;
+  }
+  const int want = env_int("DMX_CTAS_PER_SM", 0);   // tuning knob: resident CTAs per SM (0 = all that fit)
+  if (want > 0 && want < occ) occ = want;
+  const int64_t ntiles = (P + plan.tile - 1) / plan.tile;
+  plan.grid = (int)std::min<int64_t>((int64_t)prop.multiProcessorCount * occ, ntiles);
+  h->plan = plan;
+
+  // Chunks: each CTA owns a contiguous, balanced range of tiles, cut every `chunk_tiles`
+  // tiles so that fp32 per-thread partials stay short. The cut is a function of (P, tile,
+  // grid) only, so results are reproducible on a given device.
+  const int chunk_tiles = std::max(1, env_int("DMX_CHUNK_TILES", 32));
+  std::vector<int32_t> cta_chunk0(plan.grid + 1), chunk_tile0, chunk_seg0, chunk_slot0;
+  for (int b = 0; b < plan.grid; ++b) {
+    const int64_t t0 = ntiles * b / plan.grid, t1 = ntiles * (b + 1) / plan.grid;
+    cta_chunk0[b] = (int32_t)chunk_tile0.size();
+    for (int64_t t = t0; t < t1; t += chunk_tiles) chunk_tile0.push_back((int32_t)t);
+  }
+  cta_chunk0[plan.grid] = (int32_t)chunk_tile0.size();
+  const int nchunks = (int)chunk_tile0.size();
+  chunk_tile0.push_back((int32_t)ntiles);
+  // chunk c ends where the next chunk of the same CTA starts; CTA ranges are contiguous and
+  // in order, so chunk_tile0[c+1] is the end of chunk c everywhere.
+  chunk_seg0.resize(nchunks); chunk_slot0.resize(nchunks);
+  std::vector<int32_t> chunk_seg1(nchunks);
+  int64_t nslots = 0;
+  for (int c = 0; c < nchunks; ++c) {
+    const int64_t j0 = (int64_t)chunk_tile0[c] * plan.tile;
+    const int64_t j1 = std::min<int64_t>((int64_t)chunk_tile0[c + 1] * plan.tile, P);
+    chunk_seg0[c] = segment_of(seg_offsets, S, j0);
+    chunk_seg1[c] = segment_of(seg_offsets, S, j1 - 1);
+    chunk_slot0[c] = (int32_t)nslots;
+    nslots += chunk_seg1[c] - chunk_seg0[c] + 1;
+    if (nslots > (int64_t)1 << 30) { free_handle(h); return DMX_ERR_NOMEM; }
+  }
+  std::vector<int32_t> seg_lo(S), seg_hi(S);
+  for (int s = 0; s < S; ++s) {
+    if (seg_offsets[s] == seg_offsets[s + 1]) { seg_lo[s] = 1; seg_hi[s] = 0; continue; }
+    const int64_t ta = seg_offsets[s] / plan.tile, tb = (seg_offsets[s + 1] - 1) / plan.tile;
+    seg_lo[s] = (int32_t)(std::upper_bound(chunk_tile0.begin(), chunk_tile0.end() - 1, (int32_t)ta) - chunk_tile0.begin()) - 1;
+    seg_hi[s] = (int32_t)(std::upper_bound(chunk_tile0.begin(), chunk_tile0.end() - 1, (int32_t)tb) - chunk_tile0.begin()) - 1;
+  }
+  h->nchunks = nchunks; h->nslots = (int)nslots;
+
+  std::vector<int64_t> seg(seg_offsets, seg_offsets + S + 1);
+  bool ok = upload(seg, &h->seg_off) && upload(cta_chunk0, &h->cta_chunk0) && upload(chunk_tile0, &h->chunk_tile0) &&
+            upload(chunk_seg0, &h->chunk_seg0) && upload(chunk_slot0, &h->chunk_slot0) &&
+            upload(seg_lo, &h->seg_chunk_lo) && upload(seg_hi, &h->seg_chunk_hi);
+  ok = ok && cuda_ok(cudaMalloc((void**)&h->rows, (size_t)nchunks * (K + 2) * sizeof(float)));
+  ok = ok && cuda_ok(cudaMalloc((void**)&h->slots, (size_t)nslots * 2 * sizeof(float)));
+  ok = ok && cuda_ok(cudaMalloc((void**)&h->colsum, (size_t)(K + 2 + 2 * S) * sizeof(double)));
+  ok = ok && cuda_ok(cudaMalloc((void**)&h->flags, 2 * sizeof(unsigned)));
+  ok = ok && cuda_ok(cudaMemset(h->flags, 0, 2 * sizeof(unsigned)));
+  ok = ok && cuda_ok(cudaDeviceSynchronize());
+  if (!ok) {
+    const bool nomem = g_last_cuda == (int)cudaErrorMemoryAllocation;
+    free_handle(h);
+    return nomem ? DMX_ERR_NOMEM : DMX_ERR_CUDA;
+  }
+  *out = h;
+  return DMX_OK;
+}
+
+int dmx_state_len(const dmx_handle* h) {
+  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
+  return DMX_ST_HDR + h->K + 2 * h->S;
+}
+
+int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes, float* params,
+             float* momentum, float lr, float beta, float* prev_agg, float* out_state, void* cuda_stream) {
+  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
+  if (!grad_ptrs || !batch_sizes || !params || !momentum || !prev_agg || !out_state) return DMX_ERR_ARG;
+  const int K = h->K;
+  const size_t esz = h->dtype == DMX_BF16 ? 2 : 4;
+  const size_t gbytes = (size_t)h->P * esz, sbytes = (size_t)h->P * 4;
+  const size_t obytes = (size_t)(DMX_ST_HDR + K + 2 * h->S) * 4;
+  int64_t B = 0;
+  int pivot = 0;
+  for (int k = 0; k < K; ++k) {
+    if (!grad_ptrs[k]) return DMX_ERR_ARG;
+    if (batch_sizes[k] < 1) return DMX_ERR_BATCH;
+    B += batch_sizes[k];
+    if (batch_sizes[k] > batch_sizes[pivot]) pivot = k;
+  }
+  for (int k = 0; k < K; ++k)
+    if ((uintptr_t)grad_ptrs[k] & 15) return DMX_ERR_ALIGN;
+  if (((uintptr_t)params & 15) || ((uintptr_t)momentum & 15) || ((uintptr_t)prev_agg & 15) || ((uintptr_t)out_state & 3))
+    return DMX_ERR_ALIGN;
+  const void* st[4] = {params, momentum, prev_agg, out_state};
+  const size_t sn[4] = {sbytes, sbytes, sbytes, obytes};
+  for (int i = 0; i < 4; ++i) {
+    for (int j = i + 1; j < 4; ++j)
+      if (overlap(st[i], sn[i], st[j], sn[j])) return DMX_ERR_ARG;
+    for (int k = 0; k < K; ++k)
+      if (overlap(st[i], sn[i], grad_ptrs[k], gbytes)) return DMX_ERR_ARG;
+  }
+
+  dmx::StepArgs A;
+  dmx::FinalArgs F;
+  std::memset(&A, 0, sizeof(A));
+  std::memset(&F, 0, sizeof(F));
+  // processing order: the worker with the largest batch first (the pivot), the others in
+  // the caller's order
+  int slot = 0;
+  for (int i = -1; i < K; ++i) {
+    const int k = i < 0 ? pivot : i;
+    if (i >= 0 && k == pivot) continue;
+    A.grad[slot] = grad_ptrs[k];
+    A.w[slot] = (float)((double)batch_sizes[k] / (double)B);
+    A.bf[slot] = (float)batch_sizes[k];
+    F.orig[slot] = k;
+    F.b[slot] = (double)batch_sizes[k];
+    ++slot;
+  }
+  A.params = params; A.momentum = momentum; A.prev = prev_agg;
+  A.lr = lr; A.beta = beta; A.Bf = (float)B;
+  A.K = K; A.S = h->S; A.P = h->P;
+  A.seg_off = h->seg_off; A.cta_chunk0 = h->cta_chunk0; A.chunk_tile0 = h->chunk_tile0;
+  A.chunk_seg0 = h->chunk_seg0; A.chunk_slot0 = h->chunk_slot0;
+  A.rows = h->rows; A.slots = h->slots; A.err = h->flags + 1;
+
+  F.K = K; F.S = h->S; F.nchunks = h->nchunks; F.B = (double)B;
+  F.rows = h->rows; F.slots = h->slots; F.chunk_seg0 = h->chunk_seg0; F.chunk_slot0 = h->chunk_slot0;
+  F.seg_chunk_lo = h->seg_chunk_lo; F.seg_chunk_hi = h->seg_chunk_hi;
+  F.colsum = h->colsum; F.ticket = h->flags; F.err = h->flags + 1; F.out_state = out_state;
+
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A);
+  if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
+  const int ncols = K + 2 + 2 * h->S;
+  const int fblocks = (ncols + dmx::kFinalWarps - 1) / dmx::kFinalWarps;
+  dmx::finalize_kernel<<<fblocks, dmx::kFinalWarps * 32, 0, stream>>>(F);
+  if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
+  return DMX_OK;
+}
+
+int dmx_destroy(dmx_handle* h) {
+  if (!h) return DMX_OK;
+  if (h->magic != kMagic) return DMX_ERR_HANDLE;
+  free_handle(h);
+  return DMX_OK;
+}
+
+const char* dmx_strerror(int code) {
+  switch (code) {
+    case DMX_OK: return "ok";
+    case DMX_ERR_ARG: return "invalid argument (null pointer, size out of range, or aliasing buffers)";
+    case DMX_ERR_SEGMENTS: return "segment table must satisfy o[0]=0 <= o[1] <= ... <= o[S]=P";
+    case DMX_ERR_BATCH: return "every batch size must be >= 1";
+    case DMX_ERR_ALIGN: return "device pointers must be 16-byte aligned";
+    case DMX_ERR_NOMEM: return "out of host or device memory";
+    case DMX_ERR_CUDA: return "a CUDA runtime call failed";
+    case DMX_ERR_HANDLE: return "invalid or destroyed handle";
+    default: return "unknown dmx error code";
+  }
+}
+
+int dmx_last_cuda_error(void) { return g_last_cuda; }
+
+}  // extern "C"

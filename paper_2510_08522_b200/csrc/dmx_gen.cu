@@ -1,0 +1,115 @@
+// dmx_gen.cu — device-side fill kernels of the synthetic workloads (inputs only).
+//
+// A counter-based generator, Philox4x32-10 written from its published definition (Salmon,
+// Moraes, Dror, Shaw, SC'11): the four normals of elements 4i..4i+3 of stream (tag, c2, c3)
+// come from counter (i lo, i hi, c2, c3) under key (seed, tag), through Box-Muller on
+// u = (r + 0.5) / 2^32. The Python module workload.py holds the host twin of the integer
+// core and the recipes; this file holds none of the gradient step's arithmetic and is a
+// separate shared object from the step library.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace {
+
+struct U4 { uint32_t v[4]; };
+
+__device__ __forceinline__ U4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                            uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  U4 out; out.v[0] = c0; out.v[1] = c1; out.v[2] = c2; out.v[3] = c3;
+  return out;
+}
+
+__device__ __forceinline__ void normals4(int64_t i, uint32_t c2, uint32_t c3, uint32_t seed,
+                                         uint32_t tag, float z[4]) {
+  const U4 r = philox4x32_10((uint32_t)(i & 0xffffffff), (uint32_t)(i >> 32), c2, c3, seed, tag);
+  const float s = 2.3283064365386963e-10f;  // 2^-32
+  const float u0 = ((float)r.v[0] + 0.5f) * s, u1 = ((float)r.v[1] + 0.5f) * s;
+  const float u2 = ((float)r.v[2] + 0.5f) * s, u3 = ((float)r.v[3] + 0.5f) * s;
+  const float rad0 = sqrtf(-2.0f * logf(u0)), rad1 = sqrtf(-2.0f * logf(u2));
+  float sn, cs;
+  sincospif(2.0f * u1, &sn, &cs);
+  z[0] = rad0 * cs; z[1] = rad0 * sn;
+  sincospif(2.0f * u3, &sn, &cs);
+  z[2] = rad1 * cs; z[3] = rad1 * sn;
+}
+
+// mode 0: dst = base + scale*z (base may be null -> mean)   mode 1: dst += scale*z
+template <bool BF16>
+__global__ void fill_kernel(void* __restrict__ dst, const float* __restrict__ base, float mean,
+                            float scale, int64_t n, uint32_t seed, uint32_t tag, uint32_t c2,
+                            uint32_t c3, int accumulate) {
+  const int64_t ngroups = (n + 3) / 4;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < ngroups;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    float z[4];
+    normals4(i, c2, c3, seed, tag, z);
+    const int64_t j = 4 * i;
+    const int m = (n - j) < 4 ? (int)(n - j) : 4;
+    float v[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      float b = mean;
+      if (e < m) {
+        if (accumulate) b = static_cast<const float*>(dst)[j + e];
+        else if (base) b = base[j + e];
+      }
+      v[e] = fmaf(scale, z[e], b);
+    }
+    if (BF16) {
+      __nv_bfloat16* o = static_cast<__nv_bfloat16*>(dst);
+      for (int e = 0; e < m; ++e) o[j + e] = __float2bfloat16_rn(v[e]);
+    } else {
+      float* o = static_cast<float*>(dst);
+      if (m == 4) *reinterpret_cast<float4*>(o + j) = make_float4(v[0], v[1], v[2], v[3]);
+      else for (int e = 0; e < m; ++e) o[j + e] = v[e];
+    }
+  }
+}
+
+int launch(void* dst, const float* base, float mean, float scale, int64_t n, int bf16,
+           uint32_t seed, uint32_t tag, uint32_t c2, uint32_t c3, int accumulate, void* stream) {
+  if (!dst || n < 1) return -1;
+  if (accumulate && bf16) return -1;
+  if (!bf16 && (reinterpret_cast<uintptr_t>(dst) & 15)) return -4;
+  const int threads = 256;
+  int64_t blocks = ((n + 3) / 4 + threads - 1) / threads;
+  if (blocks > 148 * 64) blocks = 148 * 64;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (bf16) fill_kernel<true><<<(unsigned)blocks, threads, 0, st>>>(dst, base, mean, scale, n, seed, tag, c2, c3, accumulate);
+  else fill_kernel<false><<<(unsigned)blocks, threads, 0, st>>>(dst, base, mean, scale, n, seed, tag, c2, c3, accumulate);
+  return cudaGetLastError() == cudaSuccess ? 0 : -6;
+}
+
+}  // namespace
+
+extern "C" {
+
+// dst[j] = mean + std * z_j                                  (fp32, DEVICE, 16-byte aligned)
+int dmxgen_normal_fill(float* dst, int64_t n, uint32_t seed, uint32_t tag, uint32_t c2, uint32_t c3,
+                       float mean, float std, void* stream) {
+  return launch(dst, nullptr, mean, std, n, 0, seed, tag, c2, c3, 0, stream);
+}
+
+// dst[j] += std * z_j                                        (fp32, DEVICE, 16-byte aligned)
+int dmxgen_normal_add(float* dst, int64_t n, uint32_t seed, uint32_t tag, uint32_t c2, uint32_t c3,
+                      float std, void* stream) {
+  return launch(dst, nullptr, 0.f, std, n, 0, seed, tag, c2, c3, 1, stream);
+}
+
+// dst[j] = round_dtype(mu[j] + scale * z_j): one worker's gradient (dtype 0 fp32, 1 bf16)
+int dmxgen_grad_fill(void* dst, int dtype, const float* mu, int64_t n, uint32_t seed, uint32_t tag,
+                     uint32_t k, uint32_t step, float scale, void* stream) {
+  if (!mu || (dtype != 0 && dtype != 1)) return -1;
+  return launch(dst, mu, 0.f, scale, n, dtype, seed, tag, k, step, 0, stream);
+}
+
+}  // extern "C"

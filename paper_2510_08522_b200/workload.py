@@ -250,3 +250,88 @@ class HostProblem:
         if self.wl.drift:
             d = (DRIFT_STD * normals(self.wl.seed, TAG_DRIFT, 0, self.step_index, 0, self.wl.P))
             self.mu = (self.mu + d.astype(np.float32)).astype(np.float32)
+
+
+# ---------------------------------------------------------------------------------------------
+# device side: the same recipes through the fill kernels of lib/libdmx_gen.so
+
+
+_gen = None
+
+
+def gen_lib():
+    global _gen
+    if _gen is None:
+        import ctypes
+        import os
+        from . import build as _build
+        path = _build.lib_path("libdmx_gen.so")
+        if not os.path.exists(path):
+            raise RuntimeError("%s is not built; run `python -m paper_2510_08522_b200.build`" % path)
+        L = ctypes.CDLL(path)
+        vp, i32, i64, u32, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_uint32, ctypes.c_float
+        L.dmxgen_normal_fill.argtypes = [vp, i64, u32, u32, u32, u32, f32, f32, vp]
+        L.dmxgen_normal_add.argtypes = [vp, i64, u32, u32, u32, u32, f32, vp]
+        L.dmxgen_grad_fill.argtypes = [vp, i32, vp, i64, u32, u32, u32, u32, f32, vp]
+        for f in (L.dmxgen_normal_fill, L.dmxgen_normal_add, L.dmxgen_grad_fill):
+            f.restype = i32
+        _gen = L
+    return _gen
+
+
+class DeviceProblem:
+    """A workload resident on one GPU: K gradient buffers, mu, and the fp32 state
+    (params, momentum, prev_agg). `fill()` writes the current step's gradients with the fill
+    kernels; `advance()` moves to the next step (drift of mu). torch is used for memory only."""
+
+    def __init__(self, wl: Workload, device="cuda:0"):
+        import torch
+        self.torch = torch
+        self.wl = wl
+        self.device = torch.device(device)
+        self.seg = wl.segment_table()
+        P, dev = wl.P, self.device
+        gdt = torch.float32 if wl.dtype == F32 else torch.bfloat16
+        self.grads = [torch.empty(P, dtype=gdt, device=dev) for _ in range(wl.K)]
+        self.mu = torch.empty(P, dtype=torch.float32, device=dev)
+        self.params = torch.empty(P, dtype=torch.float32, device=dev)
+        self.momentum = torch.zeros(P, dtype=torch.float32, device=dev)
+        self.prev_agg = torch.zeros(P, dtype=torch.float32, device=dev)
+        self.step_index = 0
+        self.reset()
+
+    def _stream(self):
+        return self.torch.cuda.current_stream(self.device).cuda_stream
+
+    def _chk(self, rc, what):
+        if rc != 0:
+            raise RuntimeError("%s failed with %d" % (what, rc))
+
+    def reset(self):
+        wl, L = self.wl, gen_lib()
+        with self.torch.cuda.device(self.device):
+            self._chk(L.dmxgen_normal_fill(self.mu.data_ptr(), wl.P, wl.seed, TAG_MU, 0, 0, 0.0, MU_STD, self._stream()), "mu fill")
+            self._chk(L.dmxgen_normal_fill(self.params.data_ptr(), wl.P, wl.seed, TAG_THETA, 0, 0, 0.0, THETA_STD, self._stream()), "theta fill")
+        self.momentum.zero_()
+        self.prev_agg.zero_()
+        self.step_index = 0
+
+    def batch_sizes(self):
+        return self.wl.batch_sizes(self.step_index)
+
+    def fill(self):
+        """Write the gradients of the current step; returns its batch sizes."""
+        wl, L = self.wl, gen_lib()
+        scale = wl.grad_scale(self.step_index)
+        with self.torch.cuda.device(self.device):
+            for k, g in enumerate(self.grads):
+                self._chk(L.dmxgen_grad_fill(g.data_ptr(), wl.dtype, self.mu.data_ptr(), wl.P, wl.seed, TAG_NOISE, k,
+                                             self.step_index, float(scale[k]), self._stream()), "grad fill")
+        return self.batch_sizes()
+
+    def advance(self):
+        self.step_index += 1
+        if self.wl.drift:
+            with self.torch.cuda.device(self.device):
+                self._chk(gen_lib().dmxgen_normal_add(self.mu.data_ptr(), self.wl.P, self.wl.seed, TAG_DRIFT, 0,
+                                                      self.step_index, DRIFT_STD, self._stream()), "drift")

@@ -1,0 +1,142 @@
+"""Comparison rules between the CUDA path and the oracle (test infrastructure).
+
+Tolerances (from the target: aggregate and updated params max relative error <= 1e-5 for fp32
+gradients, <= 4e-3 for bf16 gradients; scalar statistics relative error <= 1e-4), with
+"relative" made well defined near zero:
+  - per-element vectors: |gpu - ref| <= tol_v * max(|ref|, cond), cond being the forward-error
+    scale of the sum that produced the element (sum_k w_k |x_k| for the aggregate, and so on);
+  - positive sums: plain relative error <= tol_s;
+  - differences (|G|^2^, <g,a>): error judged against the size of the terms (A, sqrt(A |a|^2));
+  - cosine: absolute <= tol_s;
+  - ratios (gns, sigma): tol_s scaled by the conditioning of the ratio, and only when the
+    denominator is not itself a cancelled difference.
+"""
+import numpy as np
+
+HDR = 16
+TOL_S = 1e-4
+TOL_V = {0: 1e-5, 1: 4e-3}
+
+
+def cond_vectors(grads_f32, b, params_in, momentum_in, lr, beta):
+    """Forward-error scales of g, m', theta' (float64 arrays)."""
+    w = np.asarray(b, np.float64) / float(np.sum(b))
+    cg = np.zeros(len(params_in), np.float64)
+    for k, x in enumerate(grads_f32):
+        cg += w[k] * np.abs(x.astype(np.float64))
+    cm = np.abs(float(np.float32(beta)) * momentum_in.astype(np.float64)) + cg
+    ct = np.abs(params_in.astype(np.float64)) + abs(float(np.float32(lr))) * cm
+    return cg, cm, ct
+
+
+def vec_err(gpu, ref, cond):
+    """max over elements of |gpu-ref| / max(|ref|, cond) (0/0 counts as 0)."""
+    gpu = gpu.astype(np.float64); ref = ref.astype(np.float64)
+    den = np.maximum(np.abs(ref), cond)
+    diff = np.abs(gpu - ref)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        r = np.where(den > 0, diff / den, np.where(diff == 0, 0.0, np.inf))
+    return float(r.max()) if r.size else 0.0
+
+
+def check_vectors(dtype, gpu_vecs, ref_vecs, conds, what=""):
+    tol = TOL_V[dtype]
+    errs = {}
+    for name, g, r, c in zip(("agg", "momentum", "params"), gpu_vecs, ref_vecs, conds):
+        e = vec_err(g, r, c)
+        errs[name] = e
+        assert e <= tol, "%s %s: max scaled error %.3e > %.1e" % (what, name, e, tol)
+    return errs
+
+
+def seg_scales(cg, seg, lo=0):
+    """sum_{j in s} cond_j^2 per segment, for the elements [lo, lo+len(cg)) this call covers."""
+    cs = np.concatenate([[0.0], np.cumsum(cg.astype(np.float64) ** 2)])
+    idx = np.clip(np.asarray(seg, np.int64) - lo, 0, len(cg))
+    return cs[idx[1:]] - cs[idx[:-1]]
+
+
+def check_state(gpu, ref, K, S, seg, b, what="", tol=TOL_S, seg_scale=None):
+    """Compare two out_state vectors (float32 arrays). Returns the max relative error seen.
+
+    seg_scale[s] = sum_{j in s} cond_j^2: a segment of a few elements inherits the forward
+    error of its elements (an element's g_j may be a cancelling sum), so N_s is allowed
+    2e-5 * seg_scale[s] on top of tol * N_s (fp32 arithmetic on exactly widened inputs)."""
+    gpu = gpu.astype(np.float64); ref = ref.astype(np.float64)
+    seg = np.asarray(seg)
+    worst = 0.0
+
+    def rel(i, name, scale=None, t=tol):
+        nonlocal worst
+        s = abs(ref[i]) if scale is None else scale
+        d = abs(gpu[i] - ref[i])
+        if s == 0:
+            assert d == 0, "%s %s: ref 0, gpu %r" % (what, name, gpu[i])
+            return
+        worst = max(worst, d / s)
+        assert d <= t * s, "%s %s: gpu %.9g ref %.9g rel %.3e > %.1e" % (what, name, gpu[i], ref[i], d / s, t)
+
+    B, A, trS, G2, pp = ref[0], ref[1], ref[2], ref[3], ref[7]
+    q_ref = ref[HDR:HDR + K]
+    Qw = float(np.dot(np.asarray(b, np.float64), q_ref))
+    assert gpu[0] == ref[0], "%s B_total" % what
+    if not np.all(np.isfinite(ref[:HDR + K])):
+        # non-finite data: only the flag and the finiteness pattern are compared
+        assert int(gpu[11]) & 1 and int(ref[11]) & 1, "%s non-finite flag" % what
+        assert np.array_equal(np.isfinite(gpu[HDR:HDR + K]), np.isfinite(q_ref)), "%s q finiteness" % what
+        return worst
+    rel(1, "agg_sqnorm")
+    if trS == 0 and K > 1:      # identical workers
+        assert abs(gpu[2]) <= 1e-6 * Qw / (K - 1), "%s tr_sigma should vanish: %r" % (what, gpu[2])
+    else:
+        rel(2, "tr_sigma")
+    rel(3, "g2_hat", scale=max(A, abs(G2)))
+    rel(6, "dot_prev", scale=max(np.sqrt(A * pp), abs(ref[6])) if A * pp > 0 else None)
+    rel(7, "prev_sqnorm")
+    assert abs(gpu[5] - ref[5]) <= tol, "%s cos_prev gpu %.9g ref %.9g" % (what, gpu[5], ref[5])
+    rel(10, "wmean_worker_sqnorm")
+    if G2 >= 1e-3 * A and G2 > 0:
+        rel(4, "gns", t=tol * (1 + A / G2)) if trS > 0 else None
+    if A > 0 and trS > 0:
+        rel(8, "sigma2_norm", t=2 * tol)
+        rel(9, "sigma_norm", t=2 * tol)
+    # flags: must match unless the reference sits on a threshold
+    fg, fr = int(gpu[11]), int(ref[11])
+    assert not fg & 16, "%s internal-error flag set" % what
+    mask = 1 | 4 | 8
+    if abs(G2) > tol * max(A, 1e-300):
+        mask |= 2
+    assert (fg & mask) == (fr & mask), "%s flags gpu %d ref %d" % (what, fg, fr)
+    assert np.all(gpu[12:16] == 0)
+    for k in range(K):
+        rel(HDR + k, "worker_sqnorm[%d]" % k)
+    for s in range(S):
+        empty = seg[s] == seg[s + 1]
+        iv, inn = HDR + K + s, HDR + K + S + s
+        if empty:
+            assert gpu[iv] == 0 and gpu[inn] == 0, "%s empty segment %d not zero" % (what, s)
+            continue
+        if ref[iv] == 0 and K > 1:
+            assert abs(gpu[iv]) <= 1e-6 * Qw / (K - 1), "%s seg_var[%d] should vanish" % (what, s)
+        else:
+            rel(iv, "seg_var[%d]" % s)
+        floor = 0.0 if seg_scale is None else 2e-5 * float(seg_scale[s])
+        if abs(gpu[inn] - ref[inn]) > floor:
+            rel(inn, "seg_agg_sqnorm[%d]" % s)
+    return worst
+
+
+def grads_to_host(torch, grads, dtype, lo=None, hi=None):
+    """Device gradient tensors -> numpy arrays in the oracle's storage format; second list
+    holds the values widened to float32."""
+    raw, wide = [], []
+    for g in grads:
+        t = g if lo is None else g[lo:hi]
+        if dtype == 0:
+            a = t.cpu().numpy()
+            raw.append(a); wide.append(a)
+        else:
+            a = t.view(torch.int16).cpu().numpy().view(np.uint16)
+            raw.append(a)
+            wide.append((a.astype(np.uint32) << np.uint32(16)).view(np.float32))
+    return raw, wide

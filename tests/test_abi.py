@@ -1,0 +1,87 @@
+"""The C-ABI library loads and exports every symbol include/dmx.h declares; argument checks
+that need no GPU return their codes. No compute calls here."""
+import ctypes
+import os
+import re
+
+import numpy as np
+
+import paper_2510_08522_b200 as D
+from paper_2510_08522_b200 import binding as B
+from paper_2510_08522_b200 import build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "dmx.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(dmx_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_is_built_and_exports_every_declared_symbol():
+    build.build()
+    lib = ctypes.CDLL(build.lib_path("libdmx.so"))
+    names = declared_functions()
+    assert set(B.EXPORTS) <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+    gen = ctypes.CDLL(build.lib_path("libdmx_gen.so"))
+    for n in ("dmxgen_normal_fill", "dmxgen_normal_add", "dmxgen_grad_fill"):
+        assert hasattr(gen, n)
+
+
+def test_binding_mirrors_header_constants():
+    text = open(os.path.join(ROOT, "include", "dmx.h")).read()
+    for name, val in re.findall(r"\b(DMX_[A-Z0-9_]+)\s*=\s*(-?\d+)", text):
+        py = name[4:]
+        if hasattr(B, py):
+            assert getattr(B, py) == int(val), name
+    assert B.ST_HDR == 16 and B.FLAG_INTERNAL == 16 and B.ERR_HANDLE == -7
+
+
+def test_create_rejects_bad_arguments_without_a_gpu():
+    assert D.dmx_create(0, 8, [0, 8])[0] == B.ERR_ARG
+    assert D.dmx_create(65, 8, [0, 8])[0] == B.ERR_ARG
+    assert D.dmx_create(2, 0, [0, 0])[0] == B.ERR_ARG
+    assert D.dmx_create(2, 8, [0, 8], 7)[0] == B.ERR_ARG
+    assert D.dmx_create(2, 8, [0, 7])[0] == B.ERR_SEGMENTS
+    assert D.dmx_create(2, 8, [1, 8])[0] == B.ERR_SEGMENTS
+    assert D.dmx_create(2, 8, [0, 5, 4, 8])[0] == B.ERR_SEGMENTS
+    assert B.dmx_state_len(None) == B.ERR_HANDLE
+    assert B.dmx_destroy(None) == B.OK
+    assert B.dmx_step(None, [16], [1], 16, 32, 0.1, 0.9, 48, 64) == B.ERR_HANDLE
+    for code in range(-7, 1):
+        assert D.strerror(code) and "unknown" not in D.strerror(code)
+    assert "unknown" in D.strerror(-99)
+
+
+def test_workload_tables():
+    from paper_2510_08522_b200 import workload as W
+    for wl in W.WORKLOADS:
+        seg = wl.segment_table()
+        assert seg[0] == 0 and seg[-1] == wl.P and len(seg) == wl.S + 1 and np.all(np.diff(seg) >= 1)
+        for t in (0, 1, wl.steps - 1):
+            b = wl.batch_sizes(t)
+            assert b.shape == (wl.K,) and b.min() >= 16 and b.max() <= 1024
+    seg3 = W.WORKLOADS[3].segment_table()
+    sizes = np.diff(seg3)
+    assert abs(sizes[26] / seg3[-1] - 0.65) < 1e-6 and abs(sizes[28] / seg3[-1] - 0.15) < 1e-6
+    # log-normal tables put boundaries at every residue mod 8
+    assert len(set(int(v) % 8 for v in W.WORKLOADS[4].segment_table())) == 8
+    # the generator's normals: mean 0, variance 1, streams independent
+    z = W.normals(0, W.TAG_NOISE, 1, 0, 0, 1 << 16)
+    z2 = W.normals(0, W.TAG_NOISE, 2, 0, 0, 1 << 16)
+    assert abs(z.mean()) < 0.02 and abs(z.var() - 1) < 0.02 and abs(np.corrcoef(z, z2)[0, 1]) < 0.02
+    assert np.array_equal(W.normals(0, W.TAG_NOISE, 1, 0, 5, 100), z[5:105])
+
+
+def test_philox_known_answer():
+    # Known-answer vectors of Philox4x32-10 from the Random123 distribution's kat_vectors.
+    from paper_2510_08522_b200 import workload as W
+    r = W.philox4x32(0, 0, 0, 0, 0, 0)
+    assert [int(x) for x in r] == [0x6627e8d5, 0xe169c58d, 0xbc57ac4c, 0x9b00dbd8]
+    r = W.philox4x32(0xffffffff, 0xffffffff, 0xffffffff, 0xffffffff, 0xffffffff, 0xffffffff)
+    assert [int(x) for x in r] == [0x408f276d, 0x41c83b0e, 0xa20bc7c6, 0x6d5451fd]
+    r = W.philox4x32(0x243f6a88, 0x85a308d3, 0x13198a2e, 0x03707344, 0xa4093822, 0x299f31d0)
+    assert [int(x) for x in r] == [0xd16cfe09, 0x94fdcceb, 0x5001e420, 0x24126ea1]
