@@ -1,0 +1,339 @@
+#!/usr/bin/env python
+"""Benchmark of the gradient step: `python bench.py --gpus N --steps K --warmup W`.
+
+A step is one pass of the whole hot path (fused aggregate + statistics + SGD-momentum update,
+then finalize) over one batch of synthetic gradients. Metric: achieved GB/s of algorithmic
+HBM bytes, P*(K*e + 24) per step, with steps/s beside it. Gradients of every step are
+generated on the device between the timed regions; each step is bracketed by CUDA events on
+the stream it is launched on, and the total is the sum of those regions (max over ranks).
+Inputs (>= 17 GB per step at the timed workloads) are far larger than L2, so no flush is needed.
+
+With N > 1 the path runs as N independent replicas (one process per GPU, no data-path
+collective): the job's value is N * bytes / max-over-ranks time.
+
+`--impl reference` times the CPU oracle instead (rank 0 only), on bounded samples.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "dmx_step_GBps"
+UNIT = "GB/s"
+
+
+def kernel_source_digest():
+    h = hashlib.sha256()
+    for rel in ("paper_2510_08522_b200/csrc/dmx_kernels.cuh", "paper_2510_08522_b200/csrc/dmx.cu"):
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def recorded_traffic(workload_name):
+    """DRAM bytes per launch of the fused kernel from the committed ncu capture, if the
+    kernel sources are still the ones that were captured; else None."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "ncu_traffic.json")) as f:
+            rec = json.load(f)
+        if rec.get("kernel_source_digest") != kernel_source_digest():
+            return None
+        return rec.get("traffic_bytes_per_launch", {}).get(workload_name)
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle samples during the timed region (reading only)."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, "/tmp/dmx_clocks_%d_%d.csv" % (os.getpid(), index)
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 7:
+                    continue
+                try:
+                    sm.append(float(p[0])); mx.append(float(p[1]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, p[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            os.remove(self.path)
+        except Exception:
+            pass
+        if sm:
+            # under-load samples: the upper half of the observed clocks
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profile=True):
+    """Time `steps` steps of workload `wl` on `device`. Returns a dict of local measurements."""
+    import torch
+    import paper_2510_08522_b200 as D
+    from paper_2510_08522_b200 import workload as W
+
+    torch.cuda.set_device(device)
+    dp = W.DeviceProblem(wl, device)
+    d = D.Dmx(wl.K, wl.P, dp.seg, wl.dtype)
+    out_state = torch.empty(d.state_len, dtype=torch.float32, device=device)
+    d.set_profiling(profile)
+    for _ in range(warmup):
+        b = dp.fill()
+        d.step(dp.grads, b, dp.params, dp.momentum, wl.lr, wl.beta, dp.prev_agg, out_state)
+        dp.advance()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(device.index if device.index is not None else 0)
+    if sample_clocks:
+        sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    fused, fin = [], []
+    wall0 = time.time()
+    for s in range(steps):
+        b = dp.fill()                     # untimed: next step's gradients
+        ev[s][0].record()
+        d.step(dp.grads, b, dp.params, dp.momentum, wl.lr, wl.beta, dp.prev_agg, out_state)
+        ev[s][1].record()
+        if profile:
+            a, f = d.profile()            # waits for this step
+            fused.append(a); fin.append(f)
+        dp.advance()
+    torch.cuda.synchronize()
+    wall = time.time() - wall0
+    clocks = sampler.stop() if sample_clocks else None
+    times = [e0.elapsed_time(e1) for e0, e1 in ev]
+    flags = int(out_state[11].item())
+    res = dict(total_ms=sum(times), times=times, fused_ms=fused, finalize_ms=fin, clocks=clocks, flags=flags,
+               wall_s=wall, launches=steps * d.launches_per_step)
+
+    # end to end: gradients start in pinned host memory, the state vector ends in host memory
+    if e2e_steps > 0:
+        host = []
+        try:
+            for g in dp.grads:
+                hbuf = torch.empty(g.shape, dtype=g.dtype, pin_memory=True)
+                hbuf.copy_(g)
+                host.append(hbuf)
+        except RuntimeError:
+            host = host[:1]               # not enough pinnable memory: reuse one pinned buffer K times
+        out_host = torch.empty(d.state_len, dtype=torch.float32, pin_memory=True)
+        b = dp.batch_sizes()
+        stream = torch.cuda.current_stream(device)
+        hsrc = [host[k % len(host)] for k in range(wl.K)]
+        d.step_host(hsrc, dp.grads, b, dp.params, dp.momentum, wl.lr, wl.beta, dp.prev_agg, out_state, out_host)
+        t_e2e = []
+        for _ in range(e2e_steps):
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            d.step_host(hsrc, dp.grads, b, dp.params, dp.momentum, wl.lr, wl.beta, dp.prev_agg, out_state, out_host)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            t_e2e.append(e0.elapsed_time(e1))
+        res["e2e_ms"] = sum(t_e2e) / len(t_e2e)
+        res["h2d_bytes"] = wl.K * wl.P * wl.elem_bytes
+        res["d2h_bytes"] = d.state_len * 4
+        res["e2e_launches"] = e2e_steps * d.launches_per_step
+        del host
+    d.close()
+    res["problem"] = dp
+    return res
+
+
+def oracle_sample(wl, elems, nthreads, reps=1, device=None):
+    """Time the CPU oracle, as it stands, on the first `elems` parameters of workload `wl`
+    (same structure, same generator). Returns (seconds per sample step, elems, threads)."""
+    import numpy as np
+    from oracle.dmx_oracle import Oracle
+    from paper_2510_08522_b200 import workload as W
+    sub = wl.scaled(P=min(elems, wl.P), S=min(wl.S, 64))
+    raw = None
+    try:
+        import torch
+        if torch.cuda.is_available():
+            dp = W.DeviceProblem(sub, device if device is not None else "cuda:0")
+            b = dp.fill()
+            torch.cuda.synchronize()
+            if sub.dtype == W.F32:
+                raw = [g.cpu().numpy() for g in dp.grads]
+            else:
+                raw = [g.view(torch.int16).cpu().numpy().view(np.uint16) for g in dp.grads]
+            params, mom, prev = dp.params.cpu().numpy(), dp.momentum.cpu().numpy(), dp.prev_agg.cpu().numpy()
+            seg = dp.seg
+            del dp
+    except Exception:
+        raw = None
+    if raw is None:
+        hp = W.HostProblem(sub)
+        raw, b = hp.grads()
+        params, mom, prev, seg = hp.params0.copy(), np.zeros(sub.P, np.float32), np.zeros(sub.P, np.float32), hp.seg
+    orc = Oracle(sub.K, sub.P, seg, sub.dtype)
+    ts = []
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        orc.step(raw, b, params, mom, sub.lr, sub.beta, prev, nthreads=nthreads)
+        ts.append(time.perf_counter() - t0)
+    return ts, sub
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=4, help="index into the workload table (default: the largest)")
+    ap.add_argument("--also", type=int, default=3, help="second workload reported under 'also' (-1: none)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-sample-elems", type=int, default=16 << 20)
+    args = ap.parse_args()
+
+    from paper_2510_08522_b200 import workload as W
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    wl = W.WORKLOADS[args.workload]
+    ncores = os.cpu_count() or 1
+    dtype_name = "f32"   # arithmetic type of the path: fp32 (gradients stored as fp32 or bf16)
+    config = {"workload": wl.name, "K": wl.K, "P": wl.P, "S": wl.S,
+              "grad_dtype": "bf16" if wl.dtype == W.BF16 else "f32", "bytes_per_step": wl.bytes_per_step,
+              "l2": "inputs larger than L2 (gradients regenerated between steps)", "parallelism": "replicas x%d" % args.gpus}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        elems = min(args.cpu_sample_elems // 4, wl.P)
+        ts, sub = oracle_sample(wl, elems, ncores, reps=args.warmup + args.steps)
+        ts = ts[args.warmup:]
+        sec = sum(ts) / len(ts)
+        val = sub.bytes_per_step / sec / 1e9
+        sample = "first %d of %d parameters of %s per step, all K workers; oracle as it stands, %d threads" % (
+            sub.P, wl.P, wl.name, ncores)
+        line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+                "steps_per_s_full_size_equivalent": val * 1e9 / wl.bytes_per_step,
+                "cpu_baseline": {"value": val, "unit": UNIT, "cores": ncores, "kind": "oracle", "sample": sample},
+                "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return 0
+
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the gradient step has no CPU path")
+    from paper_2510_08522_b200 import dist_util as DU
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+    DU.init(world, "nccl")
+    DU.barrier()
+    torch.cuda.synchronize()
+    res = run_workload(wl, args.steps, args.warmup, device, args.e2e_steps)
+    torch.cuda.synchronize()
+    DU.barrier()
+    total_ms = DU.max_over_ranks(res["total_ms"])
+    e2e_ms = DU.max_over_ranks(res.get("e2e_ms", 0.0))
+    flags_any = int(DU.max_over_ranks(float(res["flags"] & 16)))
+    del res["problem"]
+    torch.cuda.empty_cache()
+
+    also = None
+    if args.also >= 0 and args.also != args.workload and world == 1:
+        wl2 = W.WORKLOADS[args.also]
+        r2 = run_workload(wl2, max(3, args.steps // 2), args.warmup, device, 0, sample_clocks=False)
+        del r2["problem"]
+        torch.cuda.empty_cache()
+        ms2 = r2["total_ms"] / len(r2["times"])
+        f2 = sum(r2["fused_ms"]) / len(r2["fused_ms"])
+        peak, _ = measured_peak()
+        also = {"workload": wl2.name, "value": wl2.bytes_per_step / ms2 / 1e6, "unit": UNIT, "ms_per_step": ms2,
+                "steps_per_s": 1e3 / ms2, "bytes_per_step": wl2.bytes_per_step,
+                "roofline_frac": wl2.bytes_per_step / f2 / 1e6 / peak, "fused_kernel_ms": f2}
+
+    if rank != 0:
+        DU.finish()
+        return 0
+
+    ms_per_step = total_ms / args.steps
+    value = world * wl.bytes_per_step / ms_per_step / 1e6
+    peak, peak_kind = measured_peak()
+    fused_ms = sum(res["fused_ms"]) / len(res["fused_ms"])
+    achieved = wl.bytes_per_step / fused_ms / 1e6
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": dtype_name, "data": "synthetic", "config": config,
+            "steps_per_s": world * 1e3 / ms_per_step,
+            "frac_of_8TBps_nominal": value / world / 8000.0,
+            "clocks": res["clocks"],
+            "gpu_launches": res["launches"],
+            "kernel_ms": {"fused": fused_ms, "finalize": sum(res["finalize_ms"]) / len(res["finalize_ms"])},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": UNIT, "frac": achieved / peak,
+                         "peak_kind": "of " + peak_kind, "traffic": recorded_traffic(wl.name),
+                         "algorithmic_bytes_per_launch": wl.bytes_per_step},
+            "internal_error_flag": bool(flags_any)}
+    if "e2e_ms" in res:
+        line["e2e"] = {"value": world * wl.bytes_per_step / e2e_ms / 1e6, "unit": UNIT,
+                       "h2d_bytes_per_step": res["h2d_bytes"], "d2h_bytes_per_step": res["d2h_bytes"],
+                       "ms_per_step": e2e_ms, "steps": args.e2e_steps,
+                       "note": "gradients copied from pinned host memory every step; params, momentum and prev_agg stay resident"}
+    if also:
+        line["also"] = also
+    if world == 1:
+        ts, sub = oracle_sample(wl, args.cpu_sample_elems, ncores, reps=1, device=device)
+        line["cpu_baseline"] = {"value": sub.bytes_per_step / ts[0] / 1e9, "unit": UNIT, "cores": ncores, "kind": "oracle",
+                                "sample": "first %d of %d parameters of %s, all K workers, one step (%.2f s)" % (
+                                    sub.P, wl.P, wl.name, ts[0])}
+    print(json.dumps(line))
+    DU.finish()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -131,6 +131,37 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
              float* params, float* momentum, float lr, float beta, float* prev_agg,
              float* out_state, void* cuda_stream);
 
+/*
+ * dmx_step_host — the same step for a caller whose gradients sit in HOST memory (the end-to-end
+ * form of Algorithm 1's worker loop on one machine: gradients arrive from the workers' side of
+ * the bus, the model state stays resident on the GPU).
+ *   host_grad_ptrs  HOST array of K HOST pointers (pinned memory for full copy speed), each P
+ *                   elements of grad_dtype
+ *   staging_ptrs    HOST array of K DEVICE pointers, caller-owned staging buffers of P elements
+ *                   each, 16-byte aligned; they receive the copies and feed the step
+ *   out_state_dev   DEVICE, as out_state of dmx_step
+ *   out_state_host  HOST, dmx_state_len(h) fp32; filled before the call returns
+ * Enqueues K host-to-device copies, the step, and the device-to-host copy of the state vector
+ * on the stream, then waits for the stream (so this call, unlike dmx_step, is synchronous).
+ * Other arguments and errors as dmx_step; a failed copy returns DMX_ERR_CUDA.
+ */
+int dmx_step_host(dmx_handle* h, const void* const* host_grad_ptrs, void* const* staging_ptrs,
+                  const int32_t* batch_sizes, float* params, float* momentum, float lr, float beta,
+                  float* prev_agg, float* out_state_dev, float* out_state_host, void* cuda_stream);
+
+/*
+ * Per-kernel device timing of the steps of a handle (for benchmarks; off by default).
+ * With profiling on, each dmx_step records CUDA events on its stream before the fused pass,
+ * between the two kernels and after finalize. dmx_get_profile waits for the last step's
+ * events and returns the two durations in milliseconds. Errors: DMX_ERR_HANDLE,
+ * DMX_ERR_ARG (no step recorded, or profiling off), DMX_ERR_CUDA.
+ */
+int dmx_set_profiling(dmx_handle* h, int on);
+int dmx_get_profile(dmx_handle* h, float* fused_ms, float* finalize_ms);
+
+/* Number of kernels one dmx_step launches (2: fused pass, finalize). */
+int dmx_launches_per_step(const dmx_handle* h);
+
 /* Frees the tables and the scratch. NULL is accepted. The caller makes sure no step of
  * this handle is still running. */
 int dmx_destroy(dmx_handle* h);

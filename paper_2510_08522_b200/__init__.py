@@ -3,5 +3,6 @@
 `binding` mirrors the C ABI of include/dmx.h; `workload` holds the seeded synthetic inputs;
 `build` compiles the CUDA sources in-tree.
 """
-from .binding import (BF16, F32, Dmx, DmxError, dmx_create, dmx_destroy, dmx_last_cuda_error,  # noqa: F401
-                      dmx_state_len, dmx_step, strerror)
+from .binding import (BF16, F32, Dmx, DmxError, dmx_create, dmx_destroy, dmx_get_profile,  # noqa: F401
+                      dmx_last_cuda_error, dmx_launches_per_step, dmx_set_profiling, dmx_state_len, dmx_step,
+                      dmx_step_host, strerror)

@@ -18,7 +18,8 @@ ST_SIGMA2_NORM, ST_SIGMA_NORM, ST_WMEAN_SQNORM, ST_FLAGS = 8, 9, 10, 11
 ST_HDR = 16
 FLAG_NONFINITE, FLAG_G2_NONPOS, FLAG_COS_UNDEF, FLAG_SINGLE, FLAG_INTERNAL = 1, 2, 4, 8, 16
 
-EXPORTS = ("dmx_create", "dmx_state_len", "dmx_step", "dmx_destroy", "dmx_strerror", "dmx_last_cuda_error")
+EXPORTS = ("dmx_create", "dmx_state_len", "dmx_step", "dmx_step_host", "dmx_set_profiling", "dmx_get_profile",
+           "dmx_launches_per_step", "dmx_destroy", "dmx_strerror", "dmx_last_cuda_error")
 
 _lib = None
 
@@ -44,6 +45,14 @@ def lib():
         L.dmx_state_len.restype = i32
         L.dmx_step.argtypes = [vp, vp, vp, vp, vp, f32, f32, vp, vp, vp]
         L.dmx_step.restype = i32
+        L.dmx_step_host.argtypes = [vp, vp, vp, vp, vp, vp, f32, f32, vp, vp, vp, vp]
+        L.dmx_step_host.restype = i32
+        L.dmx_set_profiling.argtypes = [vp, i32]
+        L.dmx_set_profiling.restype = i32
+        L.dmx_get_profile.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(f32)]
+        L.dmx_get_profile.restype = i32
+        L.dmx_launches_per_step.argtypes = [vp]
+        L.dmx_launches_per_step.restype = i32
         L.dmx_destroy.argtypes = [vp]
         L.dmx_destroy.restype = i32
         L.dmx_strerror.argtypes = [i32]
@@ -78,6 +87,33 @@ def dmx_step(h, grad_ptrs, batch_sizes, params, momentum, lr, beta, prev_agg, ou
     bs = (ctypes.c_int32 * K)(*[int(b) for b in batch_sizes])
     return lib().dmx_step(h, gp, bs, int(params), int(momentum), float(lr), float(beta), int(prev_agg),
                           int(out_state), int(stream) if stream else None)
+
+
+def dmx_step_host(h, host_grad_ptrs, staging_ptrs, batch_sizes, params, momentum, lr, beta, prev_agg,
+                  out_state_dev, out_state_host, stream=0) -> int:
+    """Gradients in host memory (raw host addresses), staged into caller-owned device buffers;
+    synchronous: out_state_host (raw host address) is filled on return."""
+    K = len(host_grad_ptrs)
+    hp = (ctypes.c_void_p * K)(*[int(p) for p in host_grad_ptrs])
+    sp = (ctypes.c_void_p * K)(*[int(p) for p in staging_ptrs])
+    bs = (ctypes.c_int32 * K)(*[int(b) for b in batch_sizes])
+    return lib().dmx_step_host(h, hp, sp, bs, int(params), int(momentum), float(lr), float(beta), int(prev_agg),
+                               int(out_state_dev), int(out_state_host), int(stream) if stream else None)
+
+
+def dmx_set_profiling(h, on) -> int:
+    return lib().dmx_set_profiling(h, int(bool(on)))
+
+
+def dmx_get_profile(h):
+    """-> (code, fused_ms, finalize_ms) of the handle's last step."""
+    a, b = ctypes.c_float(), ctypes.c_float()
+    rc = lib().dmx_get_profile(h, ctypes.byref(a), ctypes.byref(b))
+    return rc, a.value, b.value
+
+
+def dmx_launches_per_step(h) -> int:
+    return lib().dmx_launches_per_step(h)
 
 
 def dmx_destroy(h) -> int:
@@ -123,6 +159,34 @@ class Dmx:
         if rc != OK:
             raise DmxError(rc, "dmx_step")
         return out_state
+
+    def step_host(self, host_grads, staging, batch_sizes, params, momentum, lr, beta, prev_agg, out_state_dev,
+                  out_state_host, stream=None):
+        """host_grads: K pinned CPU tensors; staging: K device tensors; out_state_host: pinned CPU tensor."""
+        torch = self._torch
+        if stream is None:
+            stream = torch.cuda.current_stream(params.device).cuda_stream
+        rc = dmx_step_host(self._h, [g.data_ptr() for g in host_grads], [g.data_ptr() for g in staging], batch_sizes,
+                           params.data_ptr(), momentum.data_ptr(), lr, beta, prev_agg.data_ptr(),
+                           out_state_dev.data_ptr(), out_state_host.data_ptr(), stream)
+        if rc != OK:
+            raise DmxError(rc, "dmx_step_host")
+        return out_state_host
+
+    def set_profiling(self, on=True):
+        rc = dmx_set_profiling(self._h, on)
+        if rc != OK:
+            raise DmxError(rc, "dmx_set_profiling")
+
+    def profile(self):
+        rc, a, b = dmx_get_profile(self._h)
+        if rc != OK:
+            raise DmxError(rc, "dmx_get_profile")
+        return a, b
+
+    @property
+    def launches_per_step(self):
+        return dmx_launches_per_step(self._h)
 
     def close(self):
         if getattr(self, "_h", None):

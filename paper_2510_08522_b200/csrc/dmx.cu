@@ -63,6 +63,9 @@ struct dmx_handle {
   float *rows = nullptr, *slots = nullptr;
   double* colsum = nullptr;
   unsigned* flags = nullptr;  // [0] ticket, [1] err
+  // optional per-kernel timing
+  bool profiling = false, profiled = false;
+  cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
 };
 
 namespace {
@@ -116,6 +119,8 @@ void free_handle(dmx_handle* h) {
   cudaFree(h->seg_off); cudaFree(h->cta_chunk0); cudaFree(h->chunk_tile0); cudaFree(h->chunk_seg0);
   cudaFree(h->chunk_slot0); cudaFree(h->seg_chunk_lo); cudaFree(h->seg_chunk_hi);
   cudaFree(h->rows); cudaFree(h->slots); cudaFree(h->colsum); cudaFree(h->flags);
+  for (int i = 0; i < 3; ++i)
+    if (h->ev[i]) cudaEventDestroy(h->ev[i]);
   (void)cudaGetLastError();
   h->magic = 0;
   delete h;
@@ -295,13 +300,68 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
   F.colsum = h->colsum; F.ticket = h->flags; F.err = h->flags + 1; F.out_state = out_state;
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const bool prof = h->profiling;
+  if (prof && !cuda_ok(cudaEventRecord(h->ev[0], stream))) return DMX_ERR_CUDA;
   h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A);
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
+  if (prof && !cuda_ok(cudaEventRecord(h->ev[1], stream))) return DMX_ERR_CUDA;
   const int ncols = K + 2 + 2 * h->S;
   const int fblocks = (ncols + dmx::kFinalWarps - 1) / dmx::kFinalWarps;
   dmx::finalize_kernel<<<fblocks, dmx::kFinalWarps * 32, 0, stream>>>(F);
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
+  if (prof) {
+    if (!cuda_ok(cudaEventRecord(h->ev[2], stream))) return DMX_ERR_CUDA;
+    h->profiled = true;
+  }
   return DMX_OK;
+}
+
+int dmx_step_host(dmx_handle* h, const void* const* host_grad_ptrs, void* const* staging_ptrs,
+                  const int32_t* batch_sizes, float* params, float* momentum, float lr, float beta,
+                  float* prev_agg, float* out_state_dev, float* out_state_host, void* cuda_stream) {
+  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
+  if (!host_grad_ptrs || !staging_ptrs || !out_state_host || !out_state_dev) return DMX_ERR_ARG;
+  const size_t gbytes = (size_t)h->P * (h->dtype == DMX_BF16 ? 2 : 4);
+  for (int k = 0; k < h->K; ++k) {
+    if (!host_grad_ptrs[k] || !staging_ptrs[k]) return DMX_ERR_ARG;
+    if ((uintptr_t)staging_ptrs[k] & 15) return DMX_ERR_ALIGN;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  for (int k = 0; k < h->K; ++k)
+    if (!cuda_ok(cudaMemcpyAsync(staging_ptrs[k], host_grad_ptrs[k], gbytes, cudaMemcpyHostToDevice, stream)))
+      return DMX_ERR_CUDA;
+  const int rc = dmx_step(h, (const void* const*)staging_ptrs, batch_sizes, params, momentum, lr, beta, prev_agg,
+                          out_state_dev, cuda_stream);
+  if (rc != DMX_OK) return rc;
+  const size_t obytes = (size_t)(DMX_ST_HDR + h->K + 2 * h->S) * sizeof(float);
+  if (!cuda_ok(cudaMemcpyAsync(out_state_host, out_state_dev, obytes, cudaMemcpyDeviceToHost, stream))) return DMX_ERR_CUDA;
+  if (!cuda_ok(cudaStreamSynchronize(stream))) return DMX_ERR_CUDA;
+  return DMX_OK;
+}
+
+int dmx_set_profiling(dmx_handle* h, int on) {
+  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
+  if (on) {
+    for (int i = 0; i < 3; ++i)
+      if (!h->ev[i] && !cuda_ok(cudaEventCreate(&h->ev[i]))) return DMX_ERR_CUDA;
+  }
+  h->profiling = on != 0;
+  h->profiled = false;
+  return DMX_OK;
+}
+
+int dmx_get_profile(dmx_handle* h, float* fused_ms, float* finalize_ms) {
+  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
+  if (!fused_ms || !finalize_ms || !h->profiling || !h->profiled) return DMX_ERR_ARG;
+  if (!cuda_ok(cudaEventSynchronize(h->ev[2]))) return DMX_ERR_CUDA;
+  if (!cuda_ok(cudaEventElapsedTime(fused_ms, h->ev[0], h->ev[1]))) return DMX_ERR_CUDA;
+  if (!cuda_ok(cudaEventElapsedTime(finalize_ms, h->ev[1], h->ev[2]))) return DMX_ERR_CUDA;
+  return DMX_OK;
+}
+
+int dmx_launches_per_step(const dmx_handle* h) {
+  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
+  return 2;
 }
 
 int dmx_destroy(dmx_handle* h) {
