@@ -57,10 +57,11 @@ struct dmx_handle {
   int nchunks = 0, nslots = 0;
   // device tables
   int64_t* seg_off = nullptr;
-  int32_t *cta_chunk0 = nullptr, *chunk_tile0 = nullptr, *chunk_seg0 = nullptr, *chunk_slot0 = nullptr;
-  int32_t *seg_chunk_lo = nullptr, *seg_chunk_hi = nullptr;
+  int32_t *tile_seg = nullptr, *cta_chunk0 = nullptr, *chunk_tile0 = nullptr, *chunk_ntiles = nullptr;
+  int32_t *chunk_slot0 = nullptr, *seg_ptr = nullptr, *seg_slots = nullptr;
   // device scratch
-  float *rows = nullptr, *slots = nullptr;
+  float* rows = nullptr;
+  float2* slots = nullptr;
   double* colsum = nullptr;
   unsigned* flags = nullptr;  // [0] ticket, [1] err
   // optional per-kernel timing
@@ -93,7 +94,8 @@ Plan pick_direct(int K) {
 }
 
 // Pipelined (bulk-copy ring) kernels. Ring geometry: 8 consumer warps, 4 gradient streams per
-// stage; as many stages as fit beside the double-buffered state stage.
+// 16 KB stage (smaller stages lose to the per-stage synchronisation, larger ones leave too few
+// in flight); as many stages as fit beside the double-buffered state stage.
 template <int KT, bool BF16>
 Plan pipe_plan() {
   typedef dmx::PipeCfg<KT, BF16, 8, 4, BF16 ? 10 : 12, 2> C;
@@ -116,8 +118,8 @@ Plan pick_pipe(int K) {
 
 void free_handle(dmx_handle* h) {
   if (!h) return;
-  cudaFree(h->seg_off); cudaFree(h->cta_chunk0); cudaFree(h->chunk_tile0); cudaFree(h->chunk_seg0);
-  cudaFree(h->chunk_slot0); cudaFree(h->seg_chunk_lo); cudaFree(h->seg_chunk_hi);
+  cudaFree(h->seg_off); cudaFree(h->tile_seg); cudaFree(h->cta_chunk0); cudaFree(h->chunk_tile0);
+  cudaFree(h->chunk_ntiles); cudaFree(h->chunk_slot0); cudaFree(h->seg_ptr); cudaFree(h->seg_slots);
   cudaFree(h->rows); cudaFree(h->slots); cudaFree(h->colsum); cudaFree(h->flags);
   for (int i = 0; i < 3; ++i)
     if (h->ev[i]) cudaEventDestroy(h->ev[i]);
@@ -181,48 +183,71 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   plan.grid = (int)std::min<int64_t>((int64_t)prop.multiProcessorCount * occ, ntiles);
   h->plan = plan;
 
-  // Chunks: each CTA owns a contiguous, balanced range of tiles, cut every `chunk_tiles`
+  // Tile t belongs to CTA t mod grid; a CTA's tiles are cut into chunks of `chunk_tiles`
   // tiles so that fp32 per-thread partials stay short. The cut is a function of (P, tile,
   // grid) only, so results are reproducible on a given device.
+  const int grid = plan.grid;
   const int chunk_tiles = std::max(1, env_int("DMX_CHUNK_TILES", 32));
-  std::vector<int32_t> cta_chunk0(plan.grid + 1), chunk_tile0, chunk_seg0, chunk_slot0;
-  for (int b = 0; b < plan.grid; ++b) {
-    const int64_t t0 = ntiles * b / plan.grid, t1 = ntiles * (b + 1) / plan.grid;
+  // per-tile segment table
+  std::vector<int32_t> tile_seg((size_t)ntiles);
+  {
+    int s = 0;
+    for (int64_t t = 0; t < ntiles; ++t) {
+      const int64_t j0 = t * plan.tile, j1 = std::min<int64_t>(j0 + plan.tile, P);
+      while (seg_offsets[s + 1] <= j0) ++s;
+      tile_seg[(size_t)t] = s | (seg_offsets[s + 1] < j1 && s < S - 1 ? dmx::kTileBoundaryBit : 0);
+    }
+  }
+  std::vector<int32_t> cta_chunk0(grid + 1), chunk_tile0, chunk_ntiles, chunk_slot0;
+  for (int b = 0; b < grid; ++b) {
     cta_chunk0[b] = (int32_t)chunk_tile0.size();
-    for (int64_t t = t0; t < t1; t += chunk_tiles) chunk_tile0.push_back((int32_t)t);
+    const int64_t nb = (ntiles - b + grid - 1) / grid;     // tiles b, b+grid, ...
+    for (int64_t i = 0; i < nb; i += chunk_tiles) {
+      chunk_tile0.push_back((int32_t)(b + i * grid));
+      chunk_ntiles.push_back((int32_t)std::min<int64_t>(chunk_tiles, nb - i));
+    }
   }
-  cta_chunk0[plan.grid] = (int32_t)chunk_tile0.size();
+  cta_chunk0[grid] = (int32_t)chunk_tile0.size();
   const int nchunks = (int)chunk_tile0.size();
-  chunk_tile0.push_back((int32_t)ntiles);
-  // chunk c ends where the next chunk of the same CTA starts; CTA ranges are contiguous and
-  // in order, so chunk_tile0[c+1] is the end of chunk c everywhere.
-  chunk_seg0.resize(nchunks); chunk_slot0.resize(nchunks);
-  std::vector<int32_t> chunk_seg1(nchunks);
-  int64_t nslots = 0;
+  // Enumerate, with the kernel's own rules, the (V, N) entries every chunk emits: a new entry
+  // whenever the running segment changes between tiles, at every boundary crossed inside a
+  // tile, and at the end of the chunk.
+  chunk_slot0.resize(nchunks);
+  std::vector<int32_t> slot_seg;                             // segment of every slot, in slot order
   for (int c = 0; c < nchunks; ++c) {
-    const int64_t j0 = (int64_t)chunk_tile0[c] * plan.tile;
-    const int64_t j1 = std::min<int64_t>((int64_t)chunk_tile0[c + 1] * plan.tile, P);
-    chunk_seg0[c] = segment_of(seg_offsets, S, j0);
-    chunk_seg1[c] = segment_of(seg_offsets, S, j1 - 1);
-    chunk_slot0[c] = (int32_t)nslots;
-    nslots += chunk_seg1[c] - chunk_seg0[c] + 1;
-    if (nslots > (int64_t)1 << 30) { free_handle(h); return DMX_ERR_NOMEM; }
+    chunk_slot0[c] = (int32_t)slot_seg.size();
+    int cur = -1;
+    for (int i = 0; i < chunk_ntiles[c]; ++i) {
+      const int64_t t = chunk_tile0[c] + (int64_t)i * grid;
+      const int64_t j1 = std::min<int64_t>((t + 1) * plan.tile, P);
+      const int s0 = tile_seg[(size_t)t] & (dmx::kTileBoundaryBit - 1);
+      if (s0 != cur) {
+        if (cur >= 0) slot_seg.push_back(cur);
+        cur = s0;
+      }
+      if (tile_seg[(size_t)t] & dmx::kTileBoundaryBit) {
+        while (cur < S - 1 && seg_offsets[cur + 1] < j1) { slot_seg.push_back(cur); ++cur; }
+      }
+    }
+    if (cur >= 0) slot_seg.push_back(cur);
+    if (slot_seg.size() > ((size_t)1 << 30)) { free_handle(h); return DMX_ERR_NOMEM; }
   }
-  std::vector<int32_t> seg_lo(S), seg_hi(S);
-  for (int s = 0; s < S; ++s) {
-    if (seg_offsets[s] == seg_offsets[s + 1]) { seg_lo[s] = 1; seg_hi[s] = 0; continue; }
-    const int64_t ta = seg_offsets[s] / plan.tile, tb = (seg_offsets[s + 1] - 1) / plan.tile;
-    seg_lo[s] = (int32_t)(std::upper_bound(chunk_tile0.begin(), chunk_tile0.end() - 1, (int32_t)ta) - chunk_tile0.begin()) - 1;
-    seg_hi[s] = (int32_t)(std::upper_bound(chunk_tile0.begin(), chunk_tile0.end() - 1, (int32_t)tb) - chunk_tile0.begin()) - 1;
+  const int64_t nslots = (int64_t)slot_seg.size();
+  std::vector<int32_t> seg_ptr(S + 1, 0), seg_slots((size_t)nslots);
+  for (int64_t i = 0; i < nslots; ++i) ++seg_ptr[slot_seg[(size_t)i] + 1];
+  for (int s = 0; s < S; ++s) seg_ptr[s + 1] += seg_ptr[s];
+  {
+    std::vector<int32_t> fill(seg_ptr.begin(), seg_ptr.end() - 1);
+    for (int64_t i = 0; i < nslots; ++i) seg_slots[(size_t)fill[slot_seg[(size_t)i]]++] = (int32_t)i;
   }
   h->nchunks = nchunks; h->nslots = (int)nslots;
 
   std::vector<int64_t> seg(seg_offsets, seg_offsets + S + 1);
-  bool ok = upload(seg, &h->seg_off) && upload(cta_chunk0, &h->cta_chunk0) && upload(chunk_tile0, &h->chunk_tile0) &&
-            upload(chunk_seg0, &h->chunk_seg0) && upload(chunk_slot0, &h->chunk_slot0) &&
-            upload(seg_lo, &h->seg_chunk_lo) && upload(seg_hi, &h->seg_chunk_hi);
+  bool ok = upload(seg, &h->seg_off) && upload(tile_seg, &h->tile_seg) && upload(cta_chunk0, &h->cta_chunk0) &&
+            upload(chunk_tile0, &h->chunk_tile0) && upload(chunk_ntiles, &h->chunk_ntiles) &&
+            upload(chunk_slot0, &h->chunk_slot0) && upload(seg_ptr, &h->seg_ptr) && upload(seg_slots, &h->seg_slots);
   ok = ok && cuda_ok(cudaMalloc((void**)&h->rows, (size_t)nchunks * (K + 2) * sizeof(float)));
-  ok = ok && cuda_ok(cudaMalloc((void**)&h->slots, (size_t)nslots * 2 * sizeof(float)));
+  ok = ok && cuda_ok(cudaMalloc((void**)&h->slots, (size_t)std::max<int64_t>(nslots, 1) * sizeof(float2)));
   ok = ok && cuda_ok(cudaMalloc((void**)&h->colsum, (size_t)(K + 2 + 2 * S) * sizeof(double)));
   ok = ok && cuda_ok(cudaMalloc((void**)&h->flags, 2 * sizeof(unsigned)));
   ok = ok && cuda_ok(cudaMemset(h->flags, 0, 2 * sizeof(unsigned)));
@@ -290,13 +315,13 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
   A.params = params; A.momentum = momentum; A.prev = prev_agg;
   A.lr = lr; A.beta = beta; A.Bf = (float)B;
   A.K = K; A.S = h->S; A.P = h->P;
-  A.seg_off = h->seg_off; A.cta_chunk0 = h->cta_chunk0; A.chunk_tile0 = h->chunk_tile0;
-  A.chunk_seg0 = h->chunk_seg0; A.chunk_slot0 = h->chunk_slot0;
+  A.tile_stride = h->plan.grid; A.nchunks = h->nchunks;
+  A.seg_off = h->seg_off; A.tile_seg = h->tile_seg; A.cta_chunk0 = h->cta_chunk0; A.chunk_tile0 = h->chunk_tile0;
+  A.chunk_ntiles = h->chunk_ntiles; A.chunk_slot0 = h->chunk_slot0;
   A.rows = h->rows; A.slots = h->slots; A.err = h->flags + 1;
 
   F.K = K; F.S = h->S; F.nchunks = h->nchunks; F.B = (double)B;
-  F.rows = h->rows; F.slots = h->slots; F.chunk_seg0 = h->chunk_seg0; F.chunk_slot0 = h->chunk_slot0;
-  F.seg_chunk_lo = h->seg_chunk_lo; F.seg_chunk_hi = h->seg_chunk_hi;
+  F.rows = h->rows; F.slots = h->slots; F.seg_ptr = h->seg_ptr; F.seg_slots = h->seg_slots;
   F.colsum = h->colsum; F.ticket = h->flags; F.err = h->flags + 1; F.out_state = out_state;
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -305,8 +330,8 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
   h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A);
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
   if (prof && !cuda_ok(cudaEventRecord(h->ev[1], stream))) return DMX_ERR_CUDA;
-  const int ncols = K + 2 + 2 * h->S;
-  const int fblocks = (ncols + dmx::kFinalWarps - 1) / dmx::kFinalWarps;
+  const int funits = K + 2 + h->S;   // one warp per chunk-row column and per segment
+  const int fblocks = (funits + dmx::kFinalWarps - 1) / dmx::kFinalWarps;
   dmx::finalize_kernel<<<fblocks, dmx::kFinalWarps * 32, 0, stream>>>(F);
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
   if (prof) {

@@ -8,12 +8,18 @@
 // The sums over k use the shifted one-pass form around a pivot worker (the one with the
 // largest batch): with e_k = x_k - x_pivot,  g = x_pivot + sum w_k e_k  and
 // d = sum b_k e_k^2 - B (sum w_k e_k)^2. Identical workers give d = 0 exactly, and the
-// cancellation is between noise-sized terms only.
+// cancellation is between noise-sized terms only. The arithmetic runs on pairs of fp32
+// values with the packed f32x2 instructions of sm_100 (each lane IEEE fp32, round to nearest).
 //
-// Reductions are deterministic: per-thread fp32 partials over a "chunk" of tiles, warp
-// shuffles, a fixed-order sum over the warps, one scratch row per chunk (and one scratch slot
-// per (chunk, segment) pair), then an fp64 fixed-order second level in the finalize kernel.
-// There are no floating-point atomics and no waits between CTAs.
+// Work layout. The parameter range is cut into tiles of T elements; tile t belongs to CTA
+// t mod grid, so at any moment the CTAs sweep a compact window of every stream (DRAM sees a
+// few dozen linear sweeps instead of thousands of scattered 4 KB reads). A CTA's tiles are
+// grouped into chunks of a few dozen tiles.
+//
+// Reductions are deterministic: per-thread fp32 partials over a chunk, warp shuffles, a
+// fixed-order sum over the warps, one scratch row per chunk and one scratch slot per
+// (chunk, run of tiles in one segment), then an fp64 fixed-order second level in the
+// finalize kernel. There are no floating-point atomics and no waits between CTAs.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -21,6 +27,8 @@
 namespace dmx {
 
 constexpr int kMaxK = 64;
+constexpr int kSegBuf = 32;                 // segment partials a CTA buffers in shared memory between drains
+constexpr int kTileBoundaryBit = 1 << 30;   // flag in the per-tile segment table
 
 // Arguments of one step; passed by value as a __grid_constant__ kernel parameter, so a step
 // needs no host-to-device copy. Worker arrays are in processing order (pivot first).
@@ -34,13 +42,17 @@ struct StepArgs {
   float lr, beta, Bf;
   int K, S;
   int64_t P;
+  int tile_stride;             // = grid size: a CTA's next tile is tile_stride further on
+  int nchunks;
   const int64_t* seg_off;      // S+1
+  const int32_t* tile_seg;     // ntiles: segment of the tile's first element; kTileBoundaryBit set
+                               //         when a segment boundary lies strictly inside the tile
   const int32_t* cta_chunk0;   // grid+1: chunks [cta_chunk0[b], cta_chunk0[b+1]) belong to CTA b
-  const int32_t* chunk_tile0;  // nchunks+1: tiles [chunk_tile0[c], chunk_tile0[c+1])
-  const int32_t* chunk_seg0;   // nchunks: segment holding the chunk's first element
+  const int32_t* chunk_tile0;  // nchunks: first tile of the chunk
+  const int32_t* chunk_ntiles; // nchunks: tiles in the chunk (tile0, tile0+stride, ...)
   const int32_t* chunk_slot0;  // nchunks: first (V,N) slot of the chunk
-  float* rows;                 // nchunks x (K+2): q_k..., c, pp
-  float* slots;                // nslots x 2: V partial, N partial
+  float* rows;                 // (K+2) x nchunks, one column after the other: q_k..., c, pp
+  float2* slots;               // nslots: (V partial, N partial), in the order the chunk emits them
   unsigned* err;               // set non-zero when a bounded wait gives up
 };
 
@@ -50,34 +62,52 @@ struct FinalArgs {
   double b[kMaxK];             // batch sizes, processing order
   double B;
   const float* rows;
-  const float* slots;
-  const int32_t* chunk_seg0;
-  const int32_t* chunk_slot0;
-  const int32_t* seg_chunk_lo; // S: first chunk touching segment s (lo > hi: empty segment)
-  const int32_t* seg_chunk_hi; // S
+  const float2* slots;
+  const int32_t* seg_ptr;      // S+1: slots of segment s are seg_slots[seg_ptr[s] .. seg_ptr[s+1])
+  const int32_t* seg_slots;
   double* colsum;              // K+2+2S
   unsigned* ticket;
   unsigned* err;
   float* out_state;
 };
 
-__device__ __forceinline__ float bits2f(uint32_t u) { return __uint_as_float(u); }
+typedef unsigned long long u64;
+
+// ---- packed fp32 pairs ---------------------------------------------------------------------
+__device__ __forceinline__ u64 pk(uint32_t lo, uint32_t hi) {
+  u64 r; asm("mov.b64 %0, {%1,%2};" : "=l"(r) : "r"(lo), "r"(hi)); return r;
+}
+__device__ __forceinline__ u64 pkf(float lo, float hi) { return pk(__float_as_uint(lo), __float_as_uint(hi)); }
+__device__ __forceinline__ void upk(u64 v, float& lo, float& hi) {
+  uint32_t a, b; asm("mov.b64 {%0,%1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+  lo = __uint_as_float(a); hi = __uint_as_float(b);
+}
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
+  u64 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d;
+}
+__device__ __forceinline__ u64 add2(u64 a, u64 b) {
+  u64 d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d;
+}
+__device__ __forceinline__ u64 mul2(u64 a, u64 b) {
+  u64 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d;
+}
 
 template <bool BF16> struct Elem;
 template <> struct Elem<false> { static constexpr int VEC = 4; typedef float T; };
 template <> struct Elem<true>  { static constexpr int VEC = 8; typedef uint16_t T; };
 
-// 16 bytes of gradient -> VEC fp32 values
+// 16 bytes of gradient -> VEC/2 fp32 pairs (bf16 widens exactly: its 16 bits are the top half)
 template <bool BF16>
-__device__ __forceinline__ void unpack(const uint4& r, float* x) {
+__device__ __forceinline__ void unpack2(const uint4& r, u64* x) {
   if constexpr (BF16) {
-    x[0] = bits2f(r.x << 16); x[1] = bits2f(r.x & 0xffff0000u);
-    x[2] = bits2f(r.y << 16); x[3] = bits2f(r.y & 0xffff0000u);
-    x[4] = bits2f(r.z << 16); x[5] = bits2f(r.z & 0xffff0000u);
-    x[6] = bits2f(r.w << 16); x[7] = bits2f(r.w & 0xffff0000u);
+    x[0] = pk(r.x << 16, r.x & 0xffff0000u); x[1] = pk(r.y << 16, r.y & 0xffff0000u);
+    x[2] = pk(r.z << 16, r.z & 0xffff0000u); x[3] = pk(r.w << 16, r.w & 0xffff0000u);
   } else {
-    x[0] = bits2f(r.x); x[1] = bits2f(r.y); x[2] = bits2f(r.z); x[3] = bits2f(r.w);
+    x[0] = pk(r.x, r.y); x[1] = pk(r.z, r.w);
   }
+}
+__device__ __forceinline__ void unpack4f(const uint4& r, float* x) {
+  x[0] = __uint_as_float(r.x); x[1] = __uint_as_float(r.y); x[2] = __uint_as_float(r.z); x[3] = __uint_as_float(r.w);
 }
 
 __device__ __forceinline__ uint4 ld_stream(const void* p) {
@@ -93,9 +123,10 @@ __device__ __forceinline__ void st_stream(float* p, float a, float b, float c, f
 // Per-thread running state of one tile (VEC consecutive parameters) and of the chunk.
 template <int KT, int VEC>
 struct Acc {
-  float p[VEC], s1[VEC], s2[VEC];   // pivot value, sum w e, sum b e^2
+  static constexpr int NP2 = VEC / 2;
+  u64 np[NP2], s1[NP2], s2[NP2];    // -pivot, sum w e, sum b e^2 (pairs)
   float q[KT];                      // per-worker sum of squares (chunk)
-  float c, pp, vs, ns;              // <g,a>, |a|^2, current segment's V and N partials (chunk)
+  float c, pp, vs, ns;              // <g,a>, |a|^2, current segment's V and N partials
 
   __device__ __forceinline__ void reset_chunk() {
 #pragma unroll
@@ -103,26 +134,28 @@ struct Acc {
     c = pp = vs = ns = 0.f;
   }
   // k is a compile-time constant after unrolling at every call site, so q[k] is a register.
-  __device__ __forceinline__ void add(int k, const float* x, float w, float bf) {
-    float sq = 0.f;
+  __device__ __forceinline__ void add(int k, const u64* x, float w, float bf) {
+    u64 sq = mul2(x[0], x[0]);
+#pragma unroll
+    for (int i = 1; i < NP2; ++i) sq = fma2(x[i], x[i], sq);
     if (k == 0) {
 #pragma unroll
-      for (int e = 0; e < VEC; ++e) { p[e] = x[e]; s1[e] = 0.f; s2[e] = 0.f; sq = fmaf(x[e], x[e], sq); }
+      for (int i = 0; i < NP2; ++i) { np[i] = x[i] ^ 0x8000000080000000ull; s1[i] = 0ull; s2[i] = 0ull; }
     } else {
+      const u64 w2 = pkf(w, w), b2 = pkf(bf, bf);
 #pragma unroll
-      for (int e = 0; e < VEC; ++e) {
-        const float d = x[e] - p[e];
-        s1[e] = fmaf(w, d, s1[e]);
-        s2[e] = fmaf(bf * d, d, s2[e]);
-        sq = fmaf(x[e], x[e], sq);
+      for (int i = 0; i < NP2; ++i) {
+        const u64 d = add2(x[i], np[i]);
+        s1[i] = fma2(w2, d, s1[i]);
+        s2[i] = fma2(mul2(b2, d), d, s2[i]);
       }
     }
-    q[k] += sq;
+    float lo, hi;
+    upk(sq, lo, hi);
+    q[k] += lo + hi;
   }
 };
 
-// Block-level pieces shared by both kernels. NW = number of participating warps; `bar_id`
-// and `nthreads` name the barrier the participating threads meet on.
 template <int NW>
 __device__ __forceinline__ void named_sync(int bar_id) {
   asm volatile("bar.sync %0, %1;" :: "r"(bar_id), "r"(NW * 32) : "memory");
@@ -134,59 +167,125 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-// Sum (vs, ns) over the participating warps in warp order and store the pair to `dst`.
-template <int NW>
-__device__ __forceinline__ void flush_pair(float vs, float ns, float* red, float* dst, int bar_id,
-                                           int wid, int lane) {
-  vs = warp_sum(vs); ns = warp_sum(ns);
-  named_sync<NW>(bar_id);                 // red[] free
-  if (lane == 0) { red[2 * wid] = vs; red[2 * wid + 1] = ns; }
+// Shared-memory work area of the reductions (used by the NW participating warps only).
+template <int KT, int NW>
+struct RedArea {
+  float rows[NW][KT + 2];
+  float2 seg[kSegBuf][NW];
+};
+
+// Per-chunk segment bookkeeping; identical in every participating thread.
+struct SegState {
+  int cur;      // segment the running (vs, ns) belong to; -1 before the chunk's first tile
+  int nent;     // entries emitted so far in this chunk
+  int nbuf;     // of which still buffered in shared memory
+};
+
+// Write the buffered segment partials to their slots (fixed order over the warps).
+template <int KT, int NW>
+__device__ __forceinline__ void seg_drain(RedArea<KT, NW>* R, SegState& st, float2* chunk_slots, int bar_id) {
   named_sync<NW>(bar_id);
-  if (wid == 0 && lane < 2) {
-    float t = 0.f;
+  for (int e = threadIdx.x; e < st.nbuf; e += NW * 32) {
+    float v = 0.f, n = 0.f;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) t += red[2 * w + lane];
-    dst[lane] = t;
+    for (int w = 0; w < NW; ++w) { const float2 t = R->seg[e][w]; v += t.x; n += t.y; }
+    chunk_slots[st.nent - st.nbuf + e] = make_float2(v, n);
+  }
+  named_sync<NW>(bar_id);
+  st.nbuf = 0;
+}
+
+// Close the running (vs, ns) as the next entry of the chunk: a warp reduction and one
+// shared-memory store per warp; no block barrier unless the shared buffer is full.
+template <int KT, int VEC, int NW>
+__device__ __forceinline__ void seg_entry(Acc<KT, VEC>& a, RedArea<KT, NW>* R, SegState& st, float2* chunk_slots,
+                                          int bar_id, int wid, int lane) {
+  const float v = warp_sum(a.vs), n = warp_sum(a.ns);
+  if (lane == 0) R->seg[st.nbuf][wid] = make_float2(v, n);
+  a.vs = 0.f; a.ns = 0.f;
+  ++st.nbuf; ++st.nent;
+  if (st.nbuf == kSegBuf) seg_drain<KT, NW>(R, st, chunk_slots, bar_id);
+}
+
+// Attribute the tile's per-element (d, g^2) to segments. `tseg` is the tile's table entry.
+// The host enumerates the entries of a chunk with the same rules (see build_tables).
+template <int KT, int VEC, int NW>
+__device__ __forceinline__ void segment_accumulate(Acc<KT, VEC>& a, const StepArgs& A, const float* dv,
+                                                   const float* nv, int64_t jt, int64_t tile_begin,
+                                                   int64_t tile_end, int tseg, RedArea<KT, NW>* R, SegState& st,
+                                                   float2* chunk_slots, int bar_id, int wid, int lane) {
+  const int s0 = tseg & (kTileBoundaryBit - 1);
+  if (s0 != st.cur) {
+    if (st.cur >= 0) seg_entry<KT, VEC, NW>(a, R, st, chunk_slots, bar_id, wid, lane);
+    st.cur = s0;
+  }
+  if (!(tseg & kTileBoundaryBit)) {
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) { a.vs += dv[e]; a.ns += nv[e]; }
+    return;
+  }
+  int64_t lo = tile_begin;                       // nothing below it is pending
+  int64_t next_bound = A.seg_off[st.cur + 1];
+  while (st.cur < A.S - 1 && next_bound < tile_end) {
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) {
+      const int64_t j = jt + e;
+      if (j >= lo && j < next_bound) { a.vs += dv[e]; a.ns += nv[e]; }
+    }
+    seg_entry<KT, VEC, NW>(a, R, st, chunk_slots, bar_id, wid, lane);
+    lo = next_bound;
+    ++st.cur;
+    next_bound = A.seg_off[st.cur + 1];
+  }
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) {
+    if (jt + e >= lo) { a.vs += dv[e]; a.ns += nv[e]; }
   }
 }
 
-// End of a chunk: q_k, c, pp -> its scratch row; (vs, ns) -> the slot of the current segment.
+// End of a chunk: last segment entry, drain, then q_k, c, pp -> the chunk's scratch row.
 template <int KT, int VEC, int NW>
-__device__ __forceinline__ void flush_chunk(Acc<KT, VEC>& a, int K, float* red, float* row,
-                                            float* slot, int bar_id, int wid, int lane) {
-  constexpr int NV = KT + 4;
+__device__ __forceinline__ void flush_chunk(Acc<KT, VEC>& a, const StepArgs& A, RedArea<KT, NW>* R, SegState& st,
+                                            int chunk, float2* chunk_slots, int bar_id, int wid, int lane) {
+  if (st.cur >= 0) seg_entry<KT, VEC, NW>(a, R, st, chunk_slots, bar_id, wid, lane);
+  constexpr int NV = KT + 2;
   float v[NV];
 #pragma unroll
   for (int k = 0; k < KT; ++k) v[k] = warp_sum(a.q[k]);
-  v[KT] = warp_sum(a.c); v[KT + 1] = warp_sum(a.pp); v[KT + 2] = warp_sum(a.vs); v[KT + 3] = warp_sum(a.ns);
-  named_sync<NW>(bar_id);
+  v[KT] = warp_sum(a.c); v[KT + 1] = warp_sum(a.pp);
   if (lane == 0) {
 #pragma unroll
-    for (int i = 0; i < NV; ++i) red[wid * NV + i] = v[i];
+    for (int i = 0; i < NV; ++i) R->rows[wid][i] = v[i];
   }
-  named_sync<NW>(bar_id);
+  seg_drain<KT, NW>(R, st, chunk_slots, bar_id);   // its first barrier also publishes rows[][]
   const int t = wid * 32 + lane;
   if (t < NV) {
     float s = 0.f;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) s += red[w * NV + t];
-    if (t < KT) { if (t < K) row[t] = s; }
-    else if (t < KT + 2) row[K + (t - KT)] = s;
-    else slot[t - KT - 2] = s;
+    for (int w = 0; w < NW; ++w) s += R->rows[w][t];
+    if (t < KT) { if (t < A.K) A.rows[(int64_t)t * A.nchunks + chunk] = s; }
+    else A.rows[(int64_t)(A.K + t - KT) * A.nchunks + chunk] = s;
   }
+  named_sync<NW>(bar_id);                          // rows[][] may be rewritten by the next chunk
   a.reset_chunk();
 }
 
-// Tile epilogue for one thread: aggregate, spread, update, statistics. `valid` = number of
-// this thread's elements below P (VEC for full tiles). State values th/m/pv are inputs and
-// are overwritten with the outputs (theta', m', g).
+// Tile epilogue for one thread: aggregate, spread, update, statistics. State values
+// th/m/pv are inputs and are overwritten with the outputs (theta', m', g).
 template <int KT, int VEC>
 __device__ __forceinline__ void finish_elements(Acc<KT, VEC>& a, const StepArgs& A, float* th, float* m,
                                                 float* pv, float* dv, float* nv) {
+  float p[VEC], s1[VEC], s2[VEC];
+#pragma unroll
+  for (int i = 0; i < VEC / 2; ++i) {
+    upk(a.np[i], p[2 * i], p[2 * i + 1]);
+    upk(a.s1[i], s1[2 * i], s1[2 * i + 1]);
+    upk(a.s2[i], s2[2 * i], s2[2 * i + 1]);
+  }
 #pragma unroll
   for (int e = 0; e < VEC; ++e) {
-    const float g = a.p[e] + a.s1[e];
-    dv[e] = fmaf(-A.Bf * a.s1[e], a.s1[e], a.s2[e]);
+    const float g = s1[e] - p[e];                // p holds the negated pivot
+    dv[e] = fmaf(-A.Bf * s1[e], s1[e], s2[e]);
     nv[e] = g * g;
     a.c = fmaf(g, pv[e], a.c);
     a.pp = fmaf(pv[e], pv[e], a.pp);
@@ -197,42 +296,9 @@ __device__ __forceinline__ void finish_elements(Acc<KT, VEC>& a, const StepArgs&
   }
 }
 
-// Attribute the tile's per-element (d, g^2) to segments. Uniform control flow across the
-// participating threads: cur_seg / next_bound are the same in all of them.
-template <int KT, int VEC, int NW>
-__device__ __forceinline__ void segment_accumulate(Acc<KT, VEC>& a, const StepArgs& A, const float* dv,
-                                                   const float* nv, int64_t jt, int64_t tile_begin,
-                                                   int64_t tile_end,
-                                                   int& cur_seg, int64_t& next_bound, float* red,
-                                                   int chunk_seg0, int chunk_slot0, int bar_id, int wid,
-                                                   int lane) {
-  if (next_bound >= tile_end || cur_seg >= A.S - 1) {
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) { a.vs += dv[e]; a.ns += nv[e]; }
-    return;
-  }
-  int64_t lo = tile_begin;  // nothing below it is pending
-  while (cur_seg < A.S - 1 && next_bound < tile_end) {
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) {
-      const int64_t j = jt + e;
-      if (j >= lo && j < next_bound) { a.vs += dv[e]; a.ns += nv[e]; }
-    }
-    flush_pair<NW>(a.vs, a.ns, red, A.slots + 2 * (int64_t)(chunk_slot0 + cur_seg - chunk_seg0), bar_id, wid, lane);
-    a.vs = 0.f; a.ns = 0.f;
-    lo = next_bound;
-    ++cur_seg;
-    next_bound = A.seg_off[cur_seg + 1];
-  }
-#pragma unroll
-  for (int e = 0; e < VEC; ++e) {
-    if (jt + e >= lo) { a.vs += dv[e]; a.ns += nv[e]; }
-  }
-}
-
 // ------------------------------------------------------------------------------------------
-// Direct kernel: every thread streams its own 16-byte pieces with plain vector loads, U
-// worker loads in flight at a time. Also the code path of the ragged last tile.
+// Direct tile: every thread streams its own 16-byte pieces with plain vector loads, U worker
+// loads in flight at a time. With GUARD it is the code path of the ragged last tile.
 
 template <int KT, bool BF16, bool GUARD, int U>
 __device__ __forceinline__ void direct_tile(Acc<KT, Elem<BF16>::VEC>& a, const StepArgs& A, int64_t jt,
@@ -242,21 +308,25 @@ __device__ __forceinline__ void direct_tile(Acc<KT, Elem<BF16>::VEC>& a, const S
 #pragma unroll
   for (int k0 = 0; k0 < KT; k0 += U) {
     if (k0 < A.K) {
-      float x[U][VEC];
+      u64 x[U][VEC / 2];
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         if (k0 + u < KT && k0 + u < A.K) {
           const GT* src = static_cast<const GT*>(A.grad[k0 + u]) + jt;
           if constexpr (GUARD) {
+            uint32_t bits[VEC];
 #pragma unroll
             for (int e = 0; e < VEC; ++e) {
+              bits[e] = 0u;
               if (jt + e < A.P) {
-                if constexpr (BF16) x[u][e] = bits2f((uint32_t)src[e] << 16); else x[u][e] = src[e];
-              } else x[u][e] = 0.f;
+                if constexpr (BF16) bits[e] = (uint32_t)src[e] << 16; else bits[e] = __float_as_uint(src[e]);
+              }
             }
+#pragma unroll
+            for (int i = 0; i < VEC / 2; ++i) x[u][i] = pk(bits[2 * i], bits[2 * i + 1]);
           } else {
             const uint4 r = ld_stream(src);
-            unpack<BF16>(r, x[u]);
+            unpack2<BF16>(r, x[u]);
           }
         }
       }
@@ -277,9 +347,9 @@ __device__ __forceinline__ void direct_tile(Acc<KT, Elem<BF16>::VEC>& a, const S
   } else {
 #pragma unroll
     for (int h = 0; h < VEC / 4; ++h) {
-      uint4 r = ld_stream(A.params + jt + 4 * h);   unpack<false>(r, th + 4 * h);
-      r = ld_stream(A.momentum + jt + 4 * h);       unpack<false>(r, m + 4 * h);
-      r = ld_stream(A.prev + jt + 4 * h);           unpack<false>(r, pv + 4 * h);
+      uint4 r = ld_stream(A.params + jt + 4 * h);   unpack4f(r, th + 4 * h);
+      r = ld_stream(A.momentum + jt + 4 * h);       unpack4f(r, m + 4 * h);
+      r = ld_stream(A.prev + jt + 4 * h);           unpack4f(r, pv + 4 * h);
     }
   }
   finish_elements<KT, VEC>(a, A, th, m, pv, dv, nv);
@@ -299,22 +369,29 @@ __device__ __forceinline__ void direct_tile(Acc<KT, Elem<BF16>::VEC>& a, const S
   }
 }
 
+// The ragged last tile, kept out of line so that its registers do not weigh on the main loop.
+template <int KT, bool BF16>
+__device__ __noinline__ void ragged_tile(Acc<KT, Elem<BF16>::VEC>& a, const StepArgs& A, int64_t jt, float* dv, float* nv) {
+  direct_tile<KT, BF16, true, 4>(a, A, jt, dv, nv);
+}
+
 template <int KT, bool BF16, int NW, int U>
 __global__ void __launch_bounds__(NW * 32)
 direct_kernel(const __grid_constant__ StepArgs A) {
   constexpr int VEC = Elem<BF16>::VEC;
   constexpr int T = NW * 32 * VEC;
-  __shared__ float red[NW * (KT + 4)];
+  __shared__ RedArea<KT, NW> R;
   const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
   Acc<KT, VEC> a;
   a.reset_chunk();
   const int c_begin = A.cta_chunk0[blockIdx.x], c_end = A.cta_chunk0[blockIdx.x + 1];
   for (int c = c_begin; c < c_end; ++c) {
-    const int t0 = A.chunk_tile0[c], t1 = A.chunk_tile0[c + 1];
-    const int seg0 = A.chunk_seg0[c], slot0 = A.chunk_slot0[c];
-    int cur_seg = seg0;
-    int64_t next_bound = A.seg_off[cur_seg + 1];
-    for (int t = t0; t < t1; ++t) {
+    const int t0 = A.chunk_tile0[c], nt = A.chunk_ntiles[c];
+    float2* chunk_slots = A.slots + A.chunk_slot0[c];
+    SegState st; st.cur = -1; st.nent = 0; st.nbuf = 0;
+    for (int i = 0; i < nt; ++i) {
+      const int t = t0 + i * A.tile_stride;
+      const int tseg = A.tile_seg[t];
       const int64_t tile_begin = (int64_t)t * T;
       const int64_t jt = tile_begin + (int64_t)threadIdx.x * VEC;
       int64_t tile_end = tile_begin + T;
@@ -325,10 +402,9 @@ direct_kernel(const __grid_constant__ StepArgs A) {
         tile_end = A.P;
         direct_tile<KT, BF16, true, U>(a, A, jt, dv, nv);
       }
-      segment_accumulate<KT, VEC, NW>(a, A, dv, nv, jt, tile_begin, tile_end, cur_seg, next_bound, red, seg0, slot0, 1, wid, lane);
+      segment_accumulate<KT, VEC, NW>(a, A, dv, nv, jt, tile_begin, tile_end, tseg, &R, st, chunk_slots, 1, wid, lane);
     }
-    flush_chunk<KT, VEC, NW>(a, A.K, red, A.rows + (int64_t)c * (A.K + 2),
-                             A.slots + 2 * (int64_t)(slot0 + cur_seg - seg0), 1, wid, lane);
+    flush_chunk<KT, VEC, NW>(a, A, &R, st, c, chunk_slots, 1, wid, lane);
   }
 }
 
@@ -343,24 +419,32 @@ __device__ __forceinline__ double warp_sum_d(double v) {
 
 constexpr int kFinalWarps = 8;
 
+// One warp per unit: units 0..K+1 are the columns q_k, c, pp of the chunk rows; unit K+2+s
+// is segment s (both of its sums).
 __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const __grid_constant__ FinalArgs F) {
   const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int K = F.K, S = F.S;
-  const int ncols = K + 2 + 2 * S;
-  const int col = blockIdx.x * kFinalWarps + wid;
-  if (col < ncols) {
-    double acc = 0.0;
-    if (col < K + 2) {
-      for (int c = lane; c < F.nchunks; c += 32) acc += (double)F.rows[(int64_t)c * (K + 2) + col];
-    } else {
-      const int which = (col - K - 2) >= S ? 1 : 0;
-      const int s = (col - K - 2) - which * S;
-      const int lo = F.seg_chunk_lo[s], hi = F.seg_chunk_hi[s];
-      for (int c = lo + lane; c <= hi; c += 32)
-        acc += (double)F.slots[2 * (int64_t)(F.chunk_slot0[c] + s - F.chunk_seg0[c]) + which];
+  const int unit = blockIdx.x * kFinalWarps + wid;
+  if (unit < K + 2) {
+    const float* col = F.rows + (int64_t)unit * F.nchunks;
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+    int c = lane;
+    for (; c + 96 < F.nchunks; c += 128) {
+      a0 += (double)col[c]; a1 += (double)col[c + 32]; a2 += (double)col[c + 64]; a3 += (double)col[c + 96];
     }
-    acc = warp_sum_d(acc);
-    if (lane == 0) F.colsum[col] = acc;
+    for (; c < F.nchunks; c += 32) a0 += (double)col[c];
+    const double acc = warp_sum_d((a0 + a1) + (a2 + a3));
+    if (lane == 0) F.colsum[unit] = acc;
+  } else if (unit < K + 2 + S) {
+    const int s = unit - (K + 2);
+    const int lo = F.seg_ptr[s], hi = F.seg_ptr[s + 1];
+    double v = 0.0, n = 0.0;
+    for (int i = lo + lane; i < hi; i += 32) {
+      const float2 t = F.slots[F.seg_slots[i]];
+      v += (double)t.x; n += (double)t.y;
+    }
+    v = warp_sum_d(v); n = warp_sum_d(n);
+    if (lane == 0) { F.colsum[K + 2 + s] = v; F.colsum[K + 2 + S + s] = n; }
   }
   __shared__ unsigned s_last;
   __shared__ double s_red[2][kFinalWarps];
@@ -377,7 +461,6 @@ __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const __grid
   aV = warp_sum_d(aV); aN = warp_sum_d(aN);
   if (lane == 0) { s_red[0][wid] = aV; s_red[1][wid] = aN; }
   __syncthreads();
-  const double inv = K >= 2 ? 1.0 / (double)(K - 1) : 0.0;
   float* out = F.out_state;
   for (int k = threadIdx.x; k < K; k += blockDim.x) out[16 + F.orig[k]] = (float)cs[k];
   for (int s = threadIdx.x; s < S; s += blockDim.x) {
@@ -392,7 +475,7 @@ __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const __grid
     const double c = cs[K], pp = cs[K + 1], B = F.B;
     int flags = 0;
     double trS = 0.0;
-    if (K >= 2) trS = D * inv; else flags |= 8;
+    if (K >= 2) trS = D / (double)(K - 1); else flags |= 8;
     const double G2 = A - trS / B;
     double gns = 0.0;
     if (G2 > 0.0) gns = trS / G2; else flags |= 2;
@@ -410,16 +493,12 @@ __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const __grid
   }
 }
 
-}  // namespace dmx
-
 // ------------------------------------------------------------------------------------------
-// Pipelined kernel: one producer thread streams whole tiles into a shared-memory ring with
-// bulk asynchronous copies (the TMA engine; non-tensor 1-D form, no multicast) completing on
+// Pipelined kernel: a producer warp streams whole tiles into a shared-memory ring with bulk
+// asynchronous copies (the TMA engine; non-tensor 1-D form, no multicast) completing on
 // mbarriers; CW consumer warps read 16 bytes per thread per stream from the ring and do the
 // arithmetic. Every wait is bounded; a wait that runs out raises the handle's error word and
 // the CTA drains without waiting any more.
-
-namespace dmx {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -491,9 +570,12 @@ struct PipeCfg {
   static constexpr int SSTAGE = 3 * SSLOT;
   static constexpr int RING = NSTAGE * STAGE;
   static constexpr int SRING = NSS * SSTAGE;
-  static constexpr int RED = CW * (KT + 4) * 4;
+  static constexpr int RED = (int)((sizeof(RedArea<KT, CW>) + 15) / 16 * 16);
   static constexpr int NBAR = 2 * NSTAGE + 2 * NSS;
   static constexpr size_t SMEM = (size_t)RING + SRING + RED + NBAR * 8 + 16;
+  static_assert(G >= 1 && G <= 32, "one producer lane per stream of a stage");
+  static_assert(NSTAGE <= 32 && NSS <= 32, "stage masks are 32 bits wide");
+  static_assert(SMEM <= 227 * 1024, "ring does not fit in shared memory");
 };
 
 template <class C>
@@ -503,7 +585,7 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
   extern __shared__ __align__(128) unsigned char smem[];
   const uint32_t ring = smem_u32(smem);
   const uint32_t sring = ring + C::RING;
-  float* red = reinterpret_cast<float*>(smem + C::RING + C::SRING);
+  RedArea<KT, CW>* R = reinterpret_cast<RedArea<KT, CW>*>(smem + C::RING + C::SRING);
   const uint32_t bars = sring + C::SRING + C::RED;
   volatile uint32_t* give_up = reinterpret_cast<volatile uint32_t*>(smem + C::RING + C::SRING + C::RED + C::NBAR * 8);
   // barrier i: full_g[i] = bars + 8 i ; empty_g[i] = bars + 8 (NSTAGE + i)
@@ -523,43 +605,55 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
 
   if (wid == CW) {
     // ---------------- producer ----------------
-    if (lane != 0) return;
+    // The whole warp takes part: every lane waits for the stage to be free, lane 0 arms the
+    // barrier with the byte count, then lane u issues the copy of stream u of the stage (one
+    // thread issuing every copy in turn is itself the bottleneck: each issue is a dependent
+    // chain of about a hundred cycles).
     const uint64_t pol = policy_evict_first();
     uint32_t stage = 0, phase = 0, ss = 0, sphase = 0;
+    uint32_t armed_g = 0, par_g = 0, armed_s = 0, par_s = 0;   // stages armed, and the parity of the last arming
     bool ok = true;
-    const int t_begin = A.chunk_tile0[c_begin], t_end = A.chunk_tile0[c_end];
-    for (int t = t_begin; t < t_end && ok; ++t) {
-      const int64_t tile_begin = (int64_t)t * T;
-      if (tile_begin + T > A.P) break;  // the ragged last tile is read with plain loads
-      for (int k0 = 0; k0 < A.K && ok; k0 += G) {
-        ok = mbar_wait(empty_g + 8 * stage, phase ^ 1u, give_up, A.err);
+    for (int c = c_begin; c < c_end && ok; ++c) {
+      const int t0 = A.chunk_tile0[c], nt = A.chunk_ntiles[c];
+      for (int i = 0; i < nt && ok; ++i) {
+        const int64_t tile_begin = (int64_t)(t0 + i * A.tile_stride) * T;
+        if (tile_begin + T > A.P) break;  // the ragged last tile is read with plain loads
+        for (int k0 = 0; k0 < A.K; k0 += G) {
+          ok = __all_sync(0xffffffffu, mbar_wait(empty_g + 8 * stage, phase ^ 1u, give_up, A.err));
+          if (!ok) break;
+          const int n = A.K - k0 < G ? A.K - k0 : G;
+          if (lane == 0) mbar_expect_tx(full_g + 8 * stage, (uint32_t)n * C::SLOT);
+          armed_g |= 1u << stage;
+          par_g = (par_g & ~(1u << stage)) | (phase << stage);
+          __syncwarp();
+          if (lane < n)
+            bulk_load(ring + stage * C::STAGE + lane * C::SLOT,
+                      static_cast<const unsigned char*>(A.grad[k0 + lane]) + tile_begin * ESZ, C::SLOT, full_g + 8 * stage, pol);
+          if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
+        }
         if (!ok) break;
-        const int n = A.K - k0 < G ? A.K - k0 : G;
-        mbar_expect_tx(full_g + 8 * stage, (uint32_t)n * C::SLOT);
-        for (int u = 0; u < n; ++u)
-          bulk_load(ring + stage * C::STAGE + u * C::SLOT,
-                    static_cast<const unsigned char*>(A.grad[k0 + u]) + tile_begin * ESZ, C::SLOT, full_g + 8 * stage, pol);
-        if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
+        ok = __all_sync(0xffffffffu, mbar_wait(empty_s + 8 * ss, sphase ^ 1u, give_up, A.err));
+        if (!ok) break;
+        if (lane == 0) mbar_expect_tx(full_s + 8 * ss, C::SSTAGE);
+        armed_s |= 1u << ss;
+        par_s = (par_s & ~(1u << ss)) | (sphase << ss);
+        __syncwarp();
+        if (lane < 3) {
+          const float* src = lane == 0 ? A.prev : (lane == 1 ? A.momentum : A.params);
+          bulk_load(sring + ss * C::SSTAGE + lane * C::SSLOT, src + tile_begin, C::SSLOT, full_s + 8 * ss, pol);
+        }
+        if (++ss == NSS) { ss = 0; sphase ^= 1u; }
       }
-      if (!ok) break;
-      ok = mbar_wait(empty_s + 8 * ss, sphase ^ 1u, give_up, A.err);
-      if (!ok) break;
-      mbar_expect_tx(full_s + 8 * ss, C::SSTAGE);
-      const uint32_t dst = sring + ss * C::SSTAGE;
-      bulk_load(dst, A.prev + tile_begin, C::SSLOT, full_s + 8 * ss, pol);
-      bulk_load(dst + C::SSLOT, A.momentum + tile_begin, C::SSLOT, full_s + 8 * ss, pol);
-      bulk_load(dst + 2 * C::SSLOT, A.params + tile_begin, C::SSLOT, full_s + 8 * ss, pol);
-      if (++ss == NSS) { ss = 0; sphase ^= 1u; }
     }
-    if (!ok) {
+    if (!ok && lane == 0) {
       // gave up: let the copies already issued land before the CTA's shared memory is released
       for (uint32_t i = 0; i < (uint32_t)NSTAGE; ++i) {
-        const uint32_t par = i < stage ? phase : phase ^ 1u;
-        for (uint32_t n = 0; n < kWaitLimit && !mbar_try_wait(full_g + 8 * i, par); ++n) {}
+        if (!((armed_g >> i) & 1u)) continue;
+        for (uint32_t n = 0; n < kWaitLimit && !mbar_try_wait(full_g + 8 * i, (par_g >> i) & 1u); ++n) {}
       }
       for (uint32_t i = 0; i < (uint32_t)NSS; ++i) {
-        const uint32_t par = i < ss ? sphase : sphase ^ 1u;
-        for (uint32_t n = 0; n < kWaitLimit && !mbar_try_wait(full_s + 8 * i, par); ++n) {}
+        if (!((armed_s >> i) & 1u)) continue;
+        for (uint32_t n = 0; n < kWaitLimit && !mbar_try_wait(full_s + 8 * i, (par_s >> i) & 1u); ++n) {}
       }
     }
     return;
@@ -572,11 +666,12 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
   uint32_t stage = 0, phase = 0, ss = 0, sphase = 0;
   bool ok = true;
   for (int c = c_begin; c < c_end; ++c) {
-    const int t0 = A.chunk_tile0[c], t1 = A.chunk_tile0[c + 1];
-    const int seg0 = A.chunk_seg0[c], slot0 = A.chunk_slot0[c];
-    int cur_seg = seg0;
-    int64_t next_bound = A.seg_off[cur_seg + 1];
-    for (int t = t0; t < t1; ++t) {
+    const int t0 = A.chunk_tile0[c], nt = A.chunk_ntiles[c];
+    float2* chunk_slots = A.slots + A.chunk_slot0[c];
+    SegState st; st.cur = -1; st.nent = 0; st.nbuf = 0;
+    for (int i = 0; i < nt; ++i) {
+      const int t = t0 + i * A.tile_stride;
+      const int tseg = A.tile_seg[t];          // needed only at the end of the tile: latency hidden
       const int64_t tile_begin = (int64_t)t * T;
       const int64_t jt = tile_begin + (int64_t)tid * VEC;
       int64_t tile_end = tile_begin + T;
@@ -597,8 +692,8 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
 #pragma unroll
             for (int u = 0; u < G; ++u) {
               if (s * G + u < KT && s * G + u < A.K) {
-                float x[VEC];
-                unpack<BF16>(r[u], x);
+                u64 x[VEC / 2];
+                unpack2<BF16>(r[u], x);
                 a.add(s * G + u, x, A.w[s * G + u], A.bf[s * G + u]);
               }
             }
@@ -610,9 +705,9 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
           const uint32_t src = sring + ss * C::SSTAGE + tid * (VEC * 4);
 #pragma unroll
           for (int h = 0; h < VEC / 4; ++h) {
-            uint4 r = lds128(src + 16 * h);               unpack<false>(r, pv + 4 * h);
-            r = lds128(src + C::SSLOT + 16 * h);          unpack<false>(r, m + 4 * h);
-            r = lds128(src + 2 * C::SSLOT + 16 * h);      unpack<false>(r, th + 4 * h);
+            uint4 r = lds128(src + 16 * h);               unpack4f(r, pv + 4 * h);
+            r = lds128(src + C::SSLOT + 16 * h);          unpack4f(r, m + 4 * h);
+            r = lds128(src + 2 * C::SSLOT + 16 * h);      unpack4f(r, th + 4 * h);
           }
         }
         __syncwarp();
@@ -629,12 +724,17 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
         }
       } else {
         tile_end = A.P;
-        direct_tile<KT, BF16, true, 4>(a, A, jt, dv, nv);
+        // through copies, so that only the copies (not the loop's registers) have their address taken
+        Acc<KT, VEC> a2 = a;
+        float dv2[VEC], nv2[VEC];
+        ragged_tile<KT, BF16>(a2, A, jt, dv2, nv2);
+        a = a2;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) { dv[e] = dv2[e]; nv[e] = nv2[e]; }
       }
-      segment_accumulate<KT, VEC, CW>(a, A, dv, nv, jt, tile_begin, tile_end, cur_seg, next_bound, red, seg0, slot0, 1, wid, lane);
+      segment_accumulate<KT, VEC, CW>(a, A, dv, nv, jt, tile_begin, tile_end, tseg, R, st, chunk_slots, 1, wid, lane);
     }
-    flush_chunk<KT, VEC, CW>(a, A.K, red, A.rows + (int64_t)c * (A.K + 2),
-                             A.slots + 2 * (int64_t)(slot0 + cur_seg - seg0), 1, wid, lane);
+    flush_chunk<KT, VEC, CW>(a, A, R, st, c, chunk_slots, 1, wid, lane);
   }
 }
 
