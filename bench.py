@@ -232,7 +232,8 @@ def main():
     ap.add_argument("--workload", type=int, default=4, help="index into the workload table (default: the largest)")
     ap.add_argument("--also", type=int, default=3, help="second workload reported under 'also' (-1: none)")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-sample-elems", type=int, default=16 << 20)
+    ap.add_argument("--cpu-sample-elems", type=int, default=16 << 20, help="0: skip the CPU-baseline leg")
+    ap.add_argument("--P", type=int, default=0, help="run the workload's structure at another size (profiling captures)")
     args = ap.parse_args()
 
     from paper_2510_08522_b200 import workload as W
@@ -240,6 +241,8 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     wl = W.WORKLOADS[args.workload]
+    if args.P:
+        wl = wl.scaled(P=args.P)
     ncores = os.cpu_count() or 1
     dtype_name = "f32"   # arithmetic type of the path: fp32 (gradients stored as fp32 or bf16)
     config = {"workload": wl.name, "K": wl.K, "P": wl.P, "S": wl.S,
@@ -325,7 +328,7 @@ def main():
                        "note": "gradients copied from pinned host memory every step; params, momentum and prev_agg stay resident"}
     if also:
         line["also"] = also
-    if world == 1:
+    if world == 1 and args.cpu_sample_elems > 0:
         ts, sub = oracle_sample(wl, args.cpu_sample_elems, ncores, reps=1, device=device)
         line["cpu_baseline"] = {"value": sub.bytes_per_step / ts[0] / 1e9, "unit": UNIT, "cores": ncores, "kind": "oracle",
                                 "sample": "first %d of %d parameters of %s, all K workers, one step (%.2f s)" % (

@@ -54,7 +54,7 @@ struct dmx_handle {
   int K = 0, S = 0, dtype = 0, device = 0;
   int64_t P = 0;
   Plan plan;
-  int nchunks = 0, nslots = 0;
+  int nchunks = 0, nslots = 0, tile_group = 1;
   // device tables
   int64_t* seg_off = nullptr;
   int32_t *tile_seg = nullptr, *cta_chunk0 = nullptr, *chunk_tile0 = nullptr, *chunk_ntiles = nullptr;
@@ -95,10 +95,11 @@ Plan pick_direct(int K) {
 
 // Pipelined (bulk-copy ring) kernels. Ring geometry: 8 consumer warps, 4 gradient streams per
 // 16 KB stage (smaller stages lose to the per-stage synchronisation, larger ones leave too few
-// in flight); as many stages as fit beside the double-buffered state stage.
+// in flight); as many stages as fit beside one state stage (a second state stage measured
+// 2-3 % slower on B200).
 template <int KT, bool BF16>
 Plan pipe_plan() {
-  typedef dmx::PipeCfg<KT, BF16, 8, 4, BF16 ? 10 : 12, 2> C;
+  typedef dmx::PipeCfg<KT, BF16, 8, 4, BF16 ? 11 : 12, 1> C;
   Plan p;
   p.kernel = dmx::pipe_kernel<C>;
   p.threads = C::THREADS;
@@ -180,14 +181,17 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   const int want = env_int("DMX_CTAS_PER_SM", 0);   // tuning knob: resident CTAs per SM (0 = all that fit)
   if (want > 0 && want < occ) occ = want;
   const int64_t ntiles = (P + plan.tile - 1) / plan.tile;
-  plan.grid = (int)std::min<int64_t>((int64_t)prop.multiProcessorCount * occ, ntiles);
+  // Tiles are dealt round robin in groups of R consecutive tiles: group g belongs to CTA
+  // g mod grid. A CTA's tiles are cut into chunks of about `DMX_CHUNK_TILES` tiles so that fp32
+  // per-thread partials stay short. The cut is a function of (P, tile, grid, R) only, so
+  // results are reproducible on a given device.
+  const int R = std::max(1, std::min(env_int("DMX_TILE_GROUP", 4), 1 << 16));   // tuning knob: tiles per group
+  const int chunk_groups = std::max(1, env_int("DMX_CHUNK_TILES", 32) / R);
+  const int64_t ngroups = (ntiles + R - 1) / R;
+  plan.grid = (int)std::min<int64_t>((int64_t)prop.multiProcessorCount * occ, ngroups);
   h->plan = plan;
-
-  // Tile t belongs to CTA t mod grid; a CTA's tiles are cut into chunks of `chunk_tiles`
-  // tiles so that fp32 per-thread partials stay short. The cut is a function of (P, tile,
-  // grid) only, so results are reproducible on a given device.
+  h->tile_group = R;
   const int grid = plan.grid;
-  const int chunk_tiles = std::max(1, env_int("DMX_CHUNK_TILES", 32));
   // per-tile segment table
   std::vector<int32_t> tile_seg((size_t)ntiles);
   {
@@ -201,10 +205,12 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   std::vector<int32_t> cta_chunk0(grid + 1), chunk_tile0, chunk_ntiles, chunk_slot0;
   for (int b = 0; b < grid; ++b) {
     cta_chunk0[b] = (int32_t)chunk_tile0.size();
-    const int64_t nb = (ntiles - b + grid - 1) / grid;     // tiles b, b+grid, ...
-    for (int64_t i = 0; i < nb; i += chunk_tiles) {
-      chunk_tile0.push_back((int32_t)(b + i * grid));
-      chunk_ntiles.push_back((int32_t)std::min<int64_t>(chunk_tiles, nb - i));
+    const int64_t nb = (ngroups - b + grid - 1) / grid;    // groups b, b+grid, ...
+    for (int64_t i = 0; i < nb; i += chunk_groups) {
+      const int64_t g0 = b + i * grid, ng = std::min<int64_t>(chunk_groups, nb - i);
+      const int64_t glast = g0 + (ng - 1) * grid;            // the last group may be cut short by ntiles
+      chunk_tile0.push_back((int32_t)(g0 * R));
+      chunk_ntiles.push_back((int32_t)((ng - 1) * R + std::min<int64_t>(R, ntiles - glast * R)));
     }
   }
   cta_chunk0[grid] = (int32_t)chunk_tile0.size();
@@ -218,7 +224,7 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
     chunk_slot0[c] = (int32_t)slot_seg.size();
     int cur = -1;
     for (int i = 0; i < chunk_ntiles[c]; ++i) {
-      const int64_t t = chunk_tile0[c] + (int64_t)i * grid;
+      const int64_t t = chunk_tile0[c] + (int64_t)(i / R) * R * grid + i % R;
       const int64_t j1 = std::min<int64_t>((t + 1) * plan.tile, P);
       const int s0 = tile_seg[(size_t)t] & (dmx::kTileBoundaryBit - 1);
       if (s0 != cur) {
@@ -315,7 +321,7 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
   A.params = params; A.momentum = momentum; A.prev = prev_agg;
   A.lr = lr; A.beta = beta; A.Bf = (float)B;
   A.K = K; A.S = h->S; A.P = h->P;
-  A.tile_stride = h->plan.grid; A.nchunks = h->nchunks;
+  A.tile_group = h->tile_group; A.group_stride = h->tile_group * h->plan.grid; A.nchunks = h->nchunks;
   A.seg_off = h->seg_off; A.tile_seg = h->tile_seg; A.cta_chunk0 = h->cta_chunk0; A.chunk_tile0 = h->chunk_tile0;
   A.chunk_ntiles = h->chunk_ntiles; A.chunk_slot0 = h->chunk_slot0;
   A.rows = h->rows; A.slots = h->slots; A.err = h->flags + 1;

@@ -11,10 +11,10 @@
 // cancellation is between noise-sized terms only. The arithmetic runs on pairs of fp32
 // values with the packed f32x2 instructions of sm_100 (each lane IEEE fp32, round to nearest).
 //
-// Work layout. The parameter range is cut into tiles of T elements; tile t belongs to CTA
-// t mod grid, so at any moment the CTAs sweep a compact window of every stream (DRAM sees a
-// few dozen linear sweeps instead of thousands of scattered 4 KB reads). A CTA's tiles are
-// grouped into chunks of a few dozen tiles.
+// Work layout. The parameter range is cut into tiles of T elements, dealt to the CTAs round
+// robin in groups of R consecutive tiles (group g belongs to CTA g mod grid), so at any moment
+// the CTAs sweep a compact window of every stream (DRAM sees a few dozen linear sweeps instead
+// of thousands of scattered 4 KB reads). A CTA's tiles are grouped into chunks of a few dozen.
 //
 // Reductions are deterministic: per-thread fp32 partials over a chunk, warp shuffles, a
 // fixed-order sum over the warps, one scratch row per chunk and one scratch slot per
@@ -42,7 +42,8 @@ struct StepArgs {
   float lr, beta, Bf;
   int K, S;
   int64_t P;
-  int tile_stride;             // = grid size: a CTA's next tile is tile_stride further on
+  int tile_group;              // R: tiles are dealt to the CTAs in groups of R consecutive tiles
+  int group_stride;            // = R * grid: distance between a CTA's successive groups
   int nchunks;
   const int64_t* seg_off;      // S+1
   const int32_t* tile_seg;     // ntiles: segment of the tile's first element; kTileBoundaryBit set
@@ -90,6 +91,12 @@ __device__ __forceinline__ u64 add2(u64 a, u64 b) {
 }
 __device__ __forceinline__ u64 mul2(u64 a, u64 b) {
   u64 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d;
+}
+
+// i-th tile of a chunk whose first tile is t0
+__device__ __forceinline__ int tile_of(const StepArgs& A, int t0, int i) {
+  const int g = i / A.tile_group;
+  return t0 + g * A.group_stride + (i - g * A.tile_group);
 }
 
 template <bool BF16> struct Elem;
@@ -390,7 +397,7 @@ direct_kernel(const __grid_constant__ StepArgs A) {
     float2* chunk_slots = A.slots + A.chunk_slot0[c];
     SegState st; st.cur = -1; st.nent = 0; st.nbuf = 0;
     for (int i = 0; i < nt; ++i) {
-      const int t = t0 + i * A.tile_stride;
+      const int t = tile_of(A, t0, i);
       const int tseg = A.tile_seg[t];
       const int64_t tile_begin = (int64_t)t * T;
       const int64_t jt = tile_begin + (int64_t)threadIdx.x * VEC;
@@ -438,12 +445,19 @@ __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const __grid
   } else if (unit < K + 2 + S) {
     const int s = unit - (K + 2);
     const int lo = F.seg_ptr[s], hi = F.seg_ptr[s + 1];
-    double v = 0.0, n = 0.0;
-    for (int i = lo + lane; i < hi; i += 32) {
+    double v = 0.0, n = 0.0, v1 = 0.0, n1 = 0.0, v2 = 0.0, n2 = 0.0, v3 = 0.0, n3 = 0.0;
+    int i = lo + lane;
+    for (; i + 96 < hi; i += 128) {          // four gathers in flight per lane; fixed summation order
+      const int i0 = F.seg_slots[i], i1 = F.seg_slots[i + 32], i2 = F.seg_slots[i + 64], i3 = F.seg_slots[i + 96];
+      const float2 t0 = F.slots[i0], t1 = F.slots[i1], t2 = F.slots[i2], t3 = F.slots[i3];
+      v += (double)t0.x; n += (double)t0.y; v1 += (double)t1.x; n1 += (double)t1.y;
+      v2 += (double)t2.x; n2 += (double)t2.y; v3 += (double)t3.x; n3 += (double)t3.y;
+    }
+    for (; i < hi; i += 32) {
       const float2 t = F.slots[F.seg_slots[i]];
       v += (double)t.x; n += (double)t.y;
     }
-    v = warp_sum_d(v); n = warp_sum_d(n);
+    v = warp_sum_d((v + v1) + (v2 + v3)); n = warp_sum_d((n + n1) + (n2 + n3));
     if (lane == 0) { F.colsum[K + 2 + s] = v; F.colsum[K + 2 + S + s] = n; }
   }
   __shared__ unsigned s_last;
@@ -616,7 +630,7 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
     for (int c = c_begin; c < c_end && ok; ++c) {
       const int t0 = A.chunk_tile0[c], nt = A.chunk_ntiles[c];
       for (int i = 0; i < nt && ok; ++i) {
-        const int64_t tile_begin = (int64_t)(t0 + i * A.tile_stride) * T;
+        const int64_t tile_begin = (int64_t)tile_of(A, t0, i) * T;
         if (tile_begin + T > A.P) break;  // the ragged last tile is read with plain loads
         for (int k0 = 0; k0 < A.K; k0 += G) {
           ok = __all_sync(0xffffffffu, mbar_wait(empty_g + 8 * stage, phase ^ 1u, give_up, A.err));
@@ -670,7 +684,7 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
     float2* chunk_slots = A.slots + A.chunk_slot0[c];
     SegState st; st.cur = -1; st.nent = 0; st.nbuf = 0;
     for (int i = 0; i < nt; ++i) {
-      const int t = t0 + i * A.tile_stride;
+      const int t = tile_of(A, t0, i);
       const int tseg = A.tile_seg[t];          // needed only at the end of the tile: latency hidden
       const int64_t tile_begin = (int64_t)t * T;
       const int64_t jt = tile_begin + (int64_t)tid * VEC;
