@@ -46,7 +46,8 @@ enum {
   DMX_ERR_ALIGN = -4,    /* a device pointer is not 16-byte aligned                        */
   DMX_ERR_NOMEM = -5,    /* host or device allocation failed                               */
   DMX_ERR_CUDA = -6,     /* a CUDA runtime call failed (see dmx_last_cuda_error)           */
-  DMX_ERR_HANDLE = -7    /* handle is NULL, destroyed or corrupt                           */
+  DMX_ERR_HANDLE = -7,   /* handle is NULL, destroyed or corrupt                           */
+  DMX_ERR_LIMIT = -8     /* problem too large for the fixed scratch of dmx_step_static     */
 };
 
 /* limits */
@@ -161,6 +162,43 @@ int dmx_get_profile(dmx_handle* h, float* fused_ms, float* finalize_ms);
 
 /* Number of kernels one dmx_step launches (2: fused pass, finalize). */
 int dmx_launches_per_step(const dmx_handle* h);
+
+/*
+ * dmx_step_static — the same step without a handle and without any allocation.
+ * (The paper has no counterpart: this entry point exists for the library's callers only.)
+ *
+ * For callers that cannot allocate device memory at the point where they need the step:
+ * code running under an allocator or memory pool that must account for every byte, a
+ * latency-critical loop that cannot afford the device-wide synchronisation a cudaMalloc may
+ * bring, or a process whose memory budget is spoken for. dmx_create allocates tables and
+ * reduction scratch; this call uses neither. Its reduction scratch is a fixed array of
+ * DMX_STATIC_SCRATCH_BYTES inside the library's device image: every GPU on which the library
+ * is loaded holds that array until the process exits.
+ *
+ *   K, P, seg_offsets, S, grad_dtype   as dmx_create (seg_offsets is HOST memory, read during
+ *                                      the call), but S <= DMX_STATIC_MAX_SEGMENTS
+ *   grad_ptrs ... cuda_stream          as dmx_step
+ *
+ * It calls no cudaMalloc, cudaFree or other allocating routine; the caller still provides
+ * every input and output buffer. It runs the plain-load kernel with one contiguous range of
+ * tiles per CTA, so it is slower than dmx_step, and its sums are taken in a different order:
+ * results agree with dmx_step to rounding, not bit for bit.
+ *
+ * The first call on each device looks up the array's device address (with that device
+ * current). Make that first call outside any stream capture.
+ * All calls on a GPU share the one array, and it keeps what the previous call left: the
+ * kernels clear what they need at the start of each call, and two calls that overlap on
+ * the same GPU (different streams, different threads) race on it. Keep calls on one GPU in
+ * stream order.
+ * Errors: as dmx_create and dmx_step, and DMX_ERR_LIMIT when S exceeds
+ * DMX_STATIC_MAX_SEGMENTS or the partial sums of this device's grid would not fit in the array.
+ */
+#define DMX_STATIC_MAX_SEGMENTS 512
+#define DMX_STATIC_SCRATCH_BYTES (1 << 20)
+int dmx_step_static(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dtype,
+                    const void* const* grad_ptrs, const int32_t* batch_sizes, float* params,
+                    float* momentum, float lr, float beta, float* prev_agg, float* out_state,
+                    void* cuda_stream);
 
 /* Frees the tables and the scratch. NULL is accepted. The caller makes sure no step of
  * this handle is still running. */

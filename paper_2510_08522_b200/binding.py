@@ -12,13 +12,14 @@ from . import build as _build
 
 F32, BF16 = 0, 1
 OK = 0
-ERR_ARG, ERR_SEGMENTS, ERR_BATCH, ERR_ALIGN, ERR_NOMEM, ERR_CUDA, ERR_HANDLE = -1, -2, -3, -4, -5, -6, -7
+ERR_ARG, ERR_SEGMENTS, ERR_BATCH, ERR_ALIGN, ERR_NOMEM, ERR_CUDA, ERR_HANDLE, ERR_LIMIT = -1, -2, -3, -4, -5, -6, -7, -8
+STATIC_MAX_SEGMENTS, STATIC_SCRATCH_BYTES = 512, 1 << 20
 ST_B_TOTAL, ST_AGG_SQNORM, ST_TR_SIGMA, ST_G2, ST_GNS, ST_COS_PREV, ST_DOT_PREV, ST_PREV_SQNORM = range(8)
 ST_SIGMA2_NORM, ST_SIGMA_NORM, ST_WMEAN_SQNORM, ST_FLAGS = 8, 9, 10, 11
 ST_HDR = 16
 FLAG_NONFINITE, FLAG_G2_NONPOS, FLAG_COS_UNDEF, FLAG_SINGLE, FLAG_INTERNAL = 1, 2, 4, 8, 16
 
-EXPORTS = ("dmx_create", "dmx_state_len", "dmx_step", "dmx_step_host", "dmx_set_profiling", "dmx_get_profile",
+EXPORTS = ("dmx_create", "dmx_state_len", "dmx_step", "dmx_step_host", "dmx_step_static", "dmx_set_profiling", "dmx_get_profile",
            "dmx_launches_per_step", "dmx_destroy", "dmx_strerror", "dmx_last_cuda_error")
 
 _lib = None
@@ -47,6 +48,8 @@ def lib():
         L.dmx_step.restype = i32
         L.dmx_step_host.argtypes = [vp, vp, vp, vp, vp, vp, f32, f32, vp, vp, vp, vp]
         L.dmx_step_host.restype = i32
+        L.dmx_step_static.argtypes = [i32, i64, vp, i32, i32, vp, vp, vp, vp, f32, f32, vp, vp, vp]
+        L.dmx_step_static.restype = i32
         L.dmx_set_profiling.argtypes = [vp, i32]
         L.dmx_set_profiling.restype = i32
         L.dmx_get_profile.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(f32)]
@@ -99,6 +102,19 @@ def dmx_step_host(h, host_grad_ptrs, staging_ptrs, batch_sizes, params, momentum
     bs = (ctypes.c_int32 * K)(*[int(b) for b in batch_sizes])
     return lib().dmx_step_host(h, hp, sp, bs, int(params), int(momentum), float(lr), float(beta), int(prev_agg),
                                int(out_state_dev), int(out_state_host), int(stream) if stream else None)
+
+
+def dmx_step_static(K, P, seg_offsets, grad_dtype, grad_ptrs, batch_sizes, params, momentum, lr, beta, prev_agg,
+                    out_state, stream=0) -> int:
+    """The step without a handle and without any allocation (fixed scratch inside the library;
+    one call at a time per GPU). Buffer arguments are raw device addresses."""
+    seg = (ctypes.c_int64 * len(seg_offsets))(*[int(v) for v in seg_offsets])
+    K = int(K)
+    gp = (ctypes.c_void_p * K)(*[int(p) for p in grad_ptrs])
+    bs = (ctypes.c_int32 * K)(*[int(b) for b in batch_sizes])
+    return lib().dmx_step_static(K, int(P), seg, len(seg_offsets) - 1, int(grad_dtype), gp, bs, int(params),
+                                 int(momentum), float(lr), float(beta), int(prev_agg), int(out_state),
+                                 int(stream) if stream else None)
 
 
 def dmx_set_profiling(h, on) -> int:

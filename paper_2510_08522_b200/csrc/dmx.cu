@@ -412,6 +412,7 @@ const char* dmx_strerror(int code) {
     case DMX_ERR_NOMEM: return "out of host or device memory";
     case DMX_ERR_CUDA: return "a CUDA runtime call failed";
     case DMX_ERR_HANDLE: return "invalid or destroyed handle";
+    case DMX_ERR_LIMIT: return "problem exceeds the fixed scratch of dmx_step_static (too many segments)";
     default: return "unknown dmx error code";
   }
 }

@@ -428,7 +428,7 @@ constexpr int kFinalWarps = 8;
 
 // One warp per unit: units 0..K+1 are the columns q_k, c, pp of the chunk rows; unit K+2+s
 // is segment s (both of its sums).
-__global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const __grid_constant__ FinalArgs F) {
+static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const __grid_constant__ FinalArgs F) {
   const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int K = F.K, S = F.S;
   const int unit = blockIdx.x * kFinalWarps + wid;
