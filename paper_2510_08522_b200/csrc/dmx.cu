@@ -58,7 +58,9 @@ struct dmx_handle {
   // device tables
   int64_t* seg_off = nullptr;
   int32_t *tile_seg = nullptr, *cta_chunk0 = nullptr, *chunk_tile0 = nullptr, *chunk_ntiles = nullptr;
-  int32_t *chunk_slot0 = nullptr, *seg_ptr = nullptr, *seg_slots = nullptr;
+  int32_t *chunk_slot0 = nullptr, *seg_slots = nullptr, *unit_lo = nullptr, *unit_hi = nullptr, *seg_unit_ptr = nullptr;
+  double2* segpart = nullptr;
+  int nunits = 0;
   // device scratch
   float* rows = nullptr;
   float2* slots = nullptr;
@@ -120,18 +122,14 @@ Plan pick_pipe(int K) {
 void free_handle(dmx_handle* h) {
   if (!h) return;
   cudaFree(h->seg_off); cudaFree(h->tile_seg); cudaFree(h->cta_chunk0); cudaFree(h->chunk_tile0);
-  cudaFree(h->chunk_ntiles); cudaFree(h->chunk_slot0); cudaFree(h->seg_ptr); cudaFree(h->seg_slots);
+  cudaFree(h->chunk_ntiles); cudaFree(h->chunk_slot0); cudaFree(h->seg_slots); cudaFree(h->unit_lo);
+  cudaFree(h->unit_hi); cudaFree(h->seg_unit_ptr); cudaFree(h->segpart);
   cudaFree(h->rows); cudaFree(h->slots); cudaFree(h->colsum); cudaFree(h->flags);
   for (int i = 0; i < 3; ++i)
     if (h->ev[i]) cudaEventDestroy(h->ev[i]);
   (void)cudaGetLastError();
   h->magic = 0;
   delete h;
-}
-
-// Segment holding element j: the unique s with o[s] <= j < o[s+1].
-int segment_of(const int64_t* o, int S, int64_t j) {
-  return (int)(std::upper_bound(o, o + S + 1, j) - o) - 1;
 }
 
 bool overlap(const void* a, size_t na, const void* b, size_t nb) {
@@ -246,15 +244,27 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
     std::vector<int32_t> fill(seg_ptr.begin(), seg_ptr.end() - 1);
     for (int64_t i = 0; i < nslots; ++i) seg_slots[(size_t)fill[slot_seg[(size_t)i]]++] = (int32_t)i;
   }
-  h->nchunks = nchunks; h->nslots = (int)nslots;
+  // finalize units: runs of at most kFinalPart slots of one segment
+  std::vector<int32_t> unit_lo, unit_hi, seg_unit_ptr(S + 1, 0);
+  for (int s = 0; s < S; ++s) {
+    seg_unit_ptr[s] = (int32_t)unit_lo.size();
+    for (int32_t lo = seg_ptr[s]; lo < seg_ptr[s + 1]; lo += dmx::kFinalPart) {
+      unit_lo.push_back(lo);
+      unit_hi.push_back(std::min<int32_t>(lo + dmx::kFinalPart, seg_ptr[s + 1]));
+    }
+  }
+  seg_unit_ptr[S] = (int32_t)unit_lo.size();
+  h->nchunks = nchunks; h->nslots = (int)nslots; h->nunits = (int)unit_lo.size();
 
   std::vector<int64_t> seg(seg_offsets, seg_offsets + S + 1);
   bool ok = upload(seg, &h->seg_off) && upload(tile_seg, &h->tile_seg) && upload(cta_chunk0, &h->cta_chunk0) &&
             upload(chunk_tile0, &h->chunk_tile0) && upload(chunk_ntiles, &h->chunk_ntiles) &&
-            upload(chunk_slot0, &h->chunk_slot0) && upload(seg_ptr, &h->seg_ptr) && upload(seg_slots, &h->seg_slots);
+            upload(chunk_slot0, &h->chunk_slot0) && upload(seg_slots, &h->seg_slots) && upload(unit_lo, &h->unit_lo) &&
+            upload(unit_hi, &h->unit_hi) && upload(seg_unit_ptr, &h->seg_unit_ptr);
+  ok = ok && cuda_ok(cudaMalloc((void**)&h->segpart, (size_t)std::max(h->nunits, 1) * sizeof(double2)));
   ok = ok && cuda_ok(cudaMalloc((void**)&h->rows, (size_t)nchunks * (K + 2) * sizeof(float)));
   ok = ok && cuda_ok(cudaMalloc((void**)&h->slots, (size_t)std::max<int64_t>(nslots, 1) * sizeof(float2)));
-  ok = ok && cuda_ok(cudaMalloc((void**)&h->colsum, (size_t)(K + 2 + 2 * S) * sizeof(double)));
+  ok = ok && cuda_ok(cudaMalloc((void**)&h->colsum, (size_t)(K + 2) * sizeof(double)));
   ok = ok && cuda_ok(cudaMalloc((void**)&h->flags, 2 * sizeof(unsigned)));
   ok = ok && cuda_ok(cudaMemset(h->flags, 0, 2 * sizeof(unsigned)));
   ok = ok && cuda_ok(cudaDeviceSynchronize());
@@ -327,7 +337,8 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
   A.rows = h->rows; A.slots = h->slots; A.err = h->flags + 1;
 
   F.K = K; F.S = h->S; F.nchunks = h->nchunks; F.B = (double)B;
-  F.rows = h->rows; F.slots = h->slots; F.seg_ptr = h->seg_ptr; F.seg_slots = h->seg_slots;
+  F.rows = h->rows; F.slots = h->slots; F.seg_slots = h->seg_slots; F.nunits = h->nunits;
+  F.unit_lo = h->unit_lo; F.unit_hi = h->unit_hi; F.seg_unit_ptr = h->seg_unit_ptr; F.segpart = h->segpart;
   F.colsum = h->colsum; F.ticket = h->flags; F.err = h->flags + 1; F.out_state = out_state;
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -336,7 +347,7 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
   h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A);
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
   if (prof && !cuda_ok(cudaEventRecord(h->ev[1], stream))) return DMX_ERR_CUDA;
-  const int funits = K + 2 + h->S;   // one warp per chunk-row column and per segment
+  const int funits = K + 2 + h->nunits;   // one warp per chunk-row column and per segment unit
   const int fblocks = (funits + dmx::kFinalWarps - 1) / dmx::kFinalWarps;
   dmx::finalize_kernel<<<fblocks, dmx::kFinalWarps * 32, 0, stream>>>(F);
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;

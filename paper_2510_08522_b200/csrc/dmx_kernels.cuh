@@ -58,15 +58,18 @@ struct StepArgs {
 };
 
 struct FinalArgs {
-  int K, S, nchunks;
+  int K, S, nchunks, nunits;
   int orig[kMaxK];             // processing slot -> caller's worker index
   double b[kMaxK];             // batch sizes, processing order
   double B;
   const float* rows;
   const float2* slots;
-  const int32_t* seg_ptr;      // S+1: slots of segment s are seg_slots[seg_ptr[s] .. seg_ptr[s+1])
-  const int32_t* seg_slots;
-  double* colsum;              // K+2+2S
+  const int32_t* seg_slots;    // slot indices grouped by segment (each group in slot order)
+  const int32_t* unit_lo;      // nunits: a unit is a run seg_slots[unit_lo .. unit_hi) of one segment,
+  const int32_t* unit_hi;      //         at most kFinalPart slots long
+  const int32_t* seg_unit_ptr; // S+1: units of segment s are [seg_unit_ptr[s], seg_unit_ptr[s+1])
+  double2* segpart;            // nunits: (V, N) of each unit
+  double* colsum;              // K+2
   unsigned* ticket;
   unsigned* err;
   float* out_state;
@@ -426,8 +429,11 @@ __device__ __forceinline__ double warp_sum_d(double v) {
 
 constexpr int kFinalWarps = 8;
 
-// One warp per unit: units 0..K+1 are the columns q_k, c, pp of the chunk rows; unit K+2+s
-// is segment s (both of its sums).
+constexpr int kFinalPart = 256;  // slots per segment unit
+
+// First level: one warp per unit. Units 0..K+1 are the columns q_k, c, pp of the chunk rows;
+// the others are runs of at most kFinalPart slots of one segment. Second level, in the last
+// block to finish: the units of each segment in order, then the derived scalars.
 static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const __grid_constant__ FinalArgs F) {
   const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int K = F.K, S = F.S;
@@ -442,9 +448,9 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
     for (; c < F.nchunks; c += 32) a0 += (double)col[c];
     const double acc = warp_sum_d((a0 + a1) + (a2 + a3));
     if (lane == 0) F.colsum[unit] = acc;
-  } else if (unit < K + 2 + S) {
-    const int s = unit - (K + 2);
-    const int lo = F.seg_ptr[s], hi = F.seg_ptr[s + 1];
+  } else if (unit < K + 2 + F.nunits) {
+    const int u = unit - (K + 2);
+    const int lo = F.unit_lo[u], hi = F.unit_hi[u];
     double v = 0.0, n = 0.0, v1 = 0.0, n1 = 0.0, v2 = 0.0, n2 = 0.0, v3 = 0.0, n3 = 0.0;
     int i = lo + lane;
     for (; i + 96 < hi; i += 128) {          // four gathers in flight per lane; fixed summation order
@@ -458,7 +464,7 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
       v += (double)t.x; n += (double)t.y;
     }
     v = warp_sum_d((v + v1) + (v2 + v3)); n = warp_sum_d((n + n1) + (n2 + n3));
-    if (lane == 0) { F.colsum[K + 2 + s] = v; F.colsum[K + 2 + S + s] = n; }
+    if (lane == 0) F.segpart[u] = make_double2(v, n);
   }
   __shared__ unsigned s_last;
   __shared__ double s_red[2][kFinalWarps];
@@ -468,24 +474,32 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  // last block: everything below reads colsum written by all blocks
-  const volatile double* cs = F.colsum;
+  // last block: everything below reads what all blocks wrote. The K+2 column sums go through
+  // shared memory so that the serial part at the end does not pay a global load per term.
+  __shared__ double cs[kMaxK + 2];
+  {
+    const volatile double* gcs = F.colsum;
+    if (threadIdx.x < K + 2) cs[threadIdx.x] = gcs[threadIdx.x];
+  }
+  const volatile double2* sp = F.segpart;
+  float* out = F.out_state;
   double aV = 0.0, aN = 0.0;
-  for (int s = threadIdx.x; s < S; s += blockDim.x) { aV += cs[K + 2 + s]; aN += cs[K + 2 + S + s]; }
+  for (int s = threadIdx.x; s < S; s += blockDim.x) {
+    double v = 0.0, n = 0.0;
+    for (int u = F.seg_unit_ptr[s]; u < F.seg_unit_ptr[s + 1]; ++u) { v += sp[u].x; n += sp[u].y; }
+    out[16 + K + s] = K >= 2 ? (float)(v / (double)(K - 1)) : 0.f;
+    out[16 + K + S + s] = (float)n;
+    aV += v; aN += n;
+  }
   aV = warp_sum_d(aV); aN = warp_sum_d(aN);
   if (lane == 0) { s_red[0][wid] = aV; s_red[1][wid] = aN; }
   __syncthreads();
-  float* out = F.out_state;
   for (int k = threadIdx.x; k < K; k += blockDim.x) out[16 + F.orig[k]] = (float)cs[k];
-  for (int s = threadIdx.x; s < S; s += blockDim.x) {
-    out[16 + K + s] = K >= 2 ? (float)(cs[K + 2 + s] / (double)(K - 1)) : 0.f;
-    out[16 + K + S + s] = (float)cs[K + 2 + S + s];
-  }
   if (threadIdx.x == 0) {
     double D = 0.0, A = 0.0, Qw = 0.0;
     for (int w = 0; w < kFinalWarps; ++w) { D += s_red[0][w]; A += s_red[1][w]; }
     bool bad = false;
-    for (int k = 0; k < K; ++k) { Qw += F.b[k] * cs[k]; bad = bad || !isfinite((float)cs[k]); }
+    for (int k = 0; k < K; ++k) { const double qk = cs[k]; Qw += F.b[k] * qk; bad = bad | !isfinite((float)qk); }
     const double c = cs[K], pp = cs[K + 1], B = F.B;
     int flags = 0;
     double trS = 0.0;
