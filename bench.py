@@ -114,7 +114,12 @@ class ClockSampler:
         return out
 
 
-def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profile=True):
+def step_bytes(wl, optimizer):
+    """Algorithmic HBM bytes of one step (Adam reads and writes one more fp32 state stream)."""
+    return wl.bytes_per_step + (8 * wl.P if optimizer == "adam" else 0)
+
+
+def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profile=True, optimizer="sgd"):
     """Time `steps` steps of workload `wl` on `device`. Returns a dict of local measurements."""
     import torch
     import paper_2510_08522_b200 as D
@@ -125,9 +130,19 @@ def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profi
     d = D.Dmx(wl.K, wl.P, dp.seg, wl.dtype)
     out_state = torch.empty(d.state_len, dtype=torch.float32, device=device)
     d.set_profiling(profile)
+    second = torch.zeros(wl.P, dtype=torch.float32, device=device) if optimizer == "adam" else None
+    tcount = [0]
+
+    def one_step(b):
+        if optimizer == "adam":
+            tcount[0] += 1
+            d.step_adam(dp.grads, b, dp.params, dp.momentum, second, 1e-3, 0.9, 0.999, 1e-8, tcount[0], dp.prev_agg, out_state)
+        else:
+            d.step(dp.grads, b, dp.params, dp.momentum, wl.lr, wl.beta, dp.prev_agg, out_state)
+
     for _ in range(warmup):
         b = dp.fill()
-        d.step(dp.grads, b, dp.params, dp.momentum, wl.lr, wl.beta, dp.prev_agg, out_state)
+        one_step(b)
         dp.advance()
     torch.cuda.synchronize()
     sampler = ClockSampler(device.index if device.index is not None else 0)
@@ -139,7 +154,7 @@ def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profi
     for s in range(steps):
         b = dp.fill()                     # untimed: next step's gradients
         ev[s][0].record()
-        d.step(dp.grads, b, dp.params, dp.momentum, wl.lr, wl.beta, dp.prev_agg, out_state)
+        one_step(b)
         ev[s][1].record()
         if profile:
             a, f = d.profile()            # waits for this step
@@ -154,7 +169,7 @@ def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profi
                wall_s=wall, launches=steps * d.launches_per_step)
 
     # end to end: gradients start in pinned host memory, the state vector ends in host memory
-    if e2e_steps > 0:
+    if e2e_steps > 0 and optimizer == "sgd":
         host = []
         try:
             for g in dp.grads:
@@ -233,6 +248,8 @@ def main():
     ap.add_argument("--also", type=int, default=3, help="second workload reported under 'also' (-1: none)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-sample-elems", type=int, default=16 << 20, help="0: skip the CPU-baseline leg")
+    ap.add_argument("--optimizer", default="sgd", choices=["sgd", "adam"],
+                    help="update applied by the step (the metric's workload uses sgd)")
     ap.add_argument("--P", type=int, default=0, help="run the workload's structure at another size (profiling captures)")
     args = ap.parse_args()
 
@@ -246,7 +263,8 @@ def main():
     ncores = os.cpu_count() or 1
     dtype_name = "f32"   # arithmetic type of the path: fp32 (gradients stored as fp32 or bf16)
     config = {"workload": wl.name, "K": wl.K, "P": wl.P, "S": wl.S,
-              "grad_dtype": "bf16" if wl.dtype == W.BF16 else "f32", "bytes_per_step": wl.bytes_per_step,
+              "grad_dtype": "bf16" if wl.dtype == W.BF16 else "f32", "optimizer": args.optimizer,
+              "bytes_per_step": step_bytes(wl, args.optimizer),
               "l2": "inputs larger than L2 (gradients regenerated between steps)", "parallelism": "replicas x%d" % args.gpus}
 
     if args.impl == "reference":
@@ -278,7 +296,7 @@ def main():
     DU.init(world, "nccl")
     DU.barrier()
     torch.cuda.synchronize()
-    res = run_workload(wl, args.steps, args.warmup, device, args.e2e_steps)
+    res = run_workload(wl, args.steps, args.warmup, device, args.e2e_steps, optimizer=args.optimizer)
     torch.cuda.synchronize()
     DU.barrier()
     total_ms = DU.max_over_ranks(res["total_ms"])
@@ -290,25 +308,27 @@ def main():
     also = None
     if args.also >= 0 and args.also != args.workload and world == 1:
         wl2 = W.WORKLOADS[args.also]
-        r2 = run_workload(wl2, max(3, args.steps // 2), args.warmup, device, 0, sample_clocks=False)
+        r2 = run_workload(wl2, max(3, args.steps // 2), args.warmup, device, 0, sample_clocks=False, optimizer=args.optimizer)
         del r2["problem"]
         torch.cuda.empty_cache()
         ms2 = r2["total_ms"] / len(r2["times"])
         f2 = sum(r2["fused_ms"]) / len(r2["fused_ms"])
         peak, _ = measured_peak()
-        also = {"workload": wl2.name, "value": wl2.bytes_per_step / ms2 / 1e6, "unit": UNIT, "ms_per_step": ms2,
-                "steps_per_s": 1e3 / ms2, "bytes_per_step": wl2.bytes_per_step,
-                "roofline_frac": wl2.bytes_per_step / f2 / 1e6 / peak, "fused_kernel_ms": f2}
+        nb2 = step_bytes(wl2, args.optimizer)
+        also = {"workload": wl2.name, "value": nb2 / ms2 / 1e6, "unit": UNIT, "ms_per_step": ms2,
+                "steps_per_s": 1e3 / ms2, "bytes_per_step": nb2,
+                "roofline_frac": nb2 / f2 / 1e6 / peak, "fused_kernel_ms": f2}
 
     if rank != 0:
         DU.finish()
         return 0
 
     ms_per_step = total_ms / args.steps
-    value = world * wl.bytes_per_step / ms_per_step / 1e6
+    nbytes = step_bytes(wl, args.optimizer)
+    value = world * nbytes / ms_per_step / 1e6
     peak, peak_kind = measured_peak()
     fused_ms = sum(res["fused_ms"]) / len(res["fused_ms"])
-    achieved = wl.bytes_per_step / fused_ms / 1e6
+    achieved = nbytes / fused_ms / 1e6
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": dtype_name, "data": "synthetic", "config": config,
@@ -318,8 +338,9 @@ def main():
             "gpu_launches": res["launches"],
             "kernel_ms": {"fused": fused_ms, "finalize": sum(res["finalize_ms"]) / len(res["finalize_ms"])},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": UNIT, "frac": achieved / peak,
-                         "peak_kind": "of " + peak_kind, "traffic": recorded_traffic(wl.name),
-                         "algorithmic_bytes_per_launch": wl.bytes_per_step},
+                         "peak_kind": "of " + peak_kind,
+                         "traffic": recorded_traffic(wl.name) if args.optimizer == "sgd" else None,
+                         "algorithmic_bytes_per_launch": nbytes},
             "internal_error_flag": bool(flags_any)}
     if "e2e_ms" in res:
         line["e2e"] = {"value": world * wl.bytes_per_step / e2e_ms / 1e6, "unit": UNIT,

@@ -133,6 +133,31 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
              float* out_state, void* cuda_stream);
 
 /*
+ * dmx_step_adam — the same pass with the Adam update in place of SGD with momentum (the paper
+ * evaluates both optimizers, Section "Workloads and Datasets", and reads sigma_norm and
+ * sigma^2_norm "for adaptive optimizers", Section "State representation"). With g the
+ * aggregate (Kingma & Ba 2015, Algorithm 1, bias-corrected form):
+ *   m' = beta1 m + (1-beta1) g          v' = beta2 v + (1-beta2) g^2
+ *   mhat = m' / (1-beta1^t)             vhat = v' / (1-beta2^t)
+ *   theta' = theta - lr * mhat / (sqrt(vhat) + eps)          prev_agg' = g
+ *   first_moment, second_moment   DEVICE, P fp32 each, 16-byte aligned, updated in place
+ *   t                             1-based step count of this call (bias correction), >= 1
+ *   0 <= beta1, beta2 < 1, eps >= 0, else DMX_ERR_ARG
+ * Everything else (arguments, errors, asynchrony, statistics) is as dmx_step. out_state has the
+ * same layout; three of its reserved entries carry the optimizer-normalised gradient statistics,
+ * with ghat_j = g_j / (sqrt(vhat_j) + eps), the aggregate in units of Adam's running scale:
+ *   out_state[12] = mean_j ghat_j     out_state[13] = var_j ghat_j (population variance over
+ *   the P parameters)                 out_state[14] = sqrt(max(out_state[13], 0))
+ * (dmx_step leaves 12..15 at 0.) This reading of "normalized variance / standard deviation
+ * of gradients" under an adaptive optimizer is this library's: the paper gives no formula.
+ */
+int dmx_step_adam(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes,
+                  float* params, float* first_moment, float* second_moment, float lr, float beta1,
+                  float beta2, float eps, int64_t t, float* prev_agg, float* out_state,
+                  void* cuda_stream);
+enum { DMX_ST_ADAM_GHAT_MEAN = 12, DMX_ST_ADAM_GHAT_VAR = 13, DMX_ST_ADAM_GHAT_STD = 14 };
+
+/*
  * dmx_step_host — the same step for a caller whose gradients sit in HOST memory (the end-to-end
  * form of Algorithm 1's worker loop on one machine: gradients arrive from the workers' side of
  * the bus, the model state stays resident on the GPU).

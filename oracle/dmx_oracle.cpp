@@ -11,7 +11,12 @@
 //     workers' gradients x_k (each a mean over b_k samples) are combined into the mean
 //     over all B = sum b_k samples, g_j = (sum_k b_k x_kj) / B, and the global model takes
 //     one SGD-momentum step m <- beta m + g, theta <- theta - lr m (Section "Workloads
-//     and Datasets" names SGD; the momentum form is the usual undampened one).
+//     and Datasets" names SGD; the momentum form is the usual undampened one), or one Adam
+//     step (the same section names ADAM; Kingma & Ba 2015, Algorithm 1):
+//     m <- b1 m + (1-b1) g, v <- b2 v + (1-b2) g^2, theta <- theta - lr mhat/(sqrt(vhat)+eps)
+//     with mhat = m/(1-b1^t), vhat = v/(1-b2^t). In Adam mode the state vector also carries
+//     mean, variance and standard deviation over the parameters of g_j/(sqrt(vhat_j)+eps),
+//     this build's reading of the "normalized" gradient statistics under an adaptive optimizer.
 //   Section "State representation", "Training Statistical Efficiency Metrics": gradient
 //     statistics, sigma_norm and sigma^2_norm; Section "RL Agent Inference Evaluation",
 //     "Batch Size Adaptation Dynamics": the gradient noise scale.
@@ -69,7 +74,7 @@ double widen(const void* base, int dtype, int64_t i) {
 
 struct Partial {
   std::vector<Sum> q;      // K
-  Sum c, pp;
+  Sum c, pp, su, su2;
   int seg_first = 0;       // V, N cover segments seg_first .. seg_first + V.size() - 1
   std::vector<Sum> V, N;
 };
@@ -84,9 +89,12 @@ struct dmxo {
   bool open = false;
   std::vector<double> b;
   double B = 0, lr = 0, beta = 0;
+  bool adam = false;       // Adam update instead of SGD with momentum (beta is then beta1)
+  double beta2 = 0, eps = 0;
+  int64_t t = 0;           // 1-based step count (bias correction)
   int64_t next = 0;        // next element expected by dmxo_range
   std::vector<Sum> q, V, N;
-  Sum c, pp;
+  Sum c, pp, su, su2;
 };
 
 namespace {
@@ -104,7 +112,7 @@ int segment_of(const dmxo& h, int64_t j) {
 
 // Elements [j0, j1) of the step; pointers address element `base`.
 void run_block(const dmxo& h, int64_t base, int64_t j0, int64_t j1, const void* const* grads,
-               float* params, float* momentum, float* prev_agg, Partial& out) {
+               float* params, float* momentum, float* second, float* prev_agg, Partial& out) {
   const int K = h.K;
   out.q.assign(K, Sum());
   out.seg_first = segment_of(h, j0);
@@ -136,11 +144,27 @@ void run_block(const dmxo& h, int64_t base, int64_t j0, int64_t j1, const void* 
     const double a = (double)prev_agg[i];
     out.c.add(g * a);
     out.pp.add(a * a);
-    // SGD with momentum
-    const double m_new = h.beta * (double)momentum[i] + g;
-    const double th_new = (double)params[i] - h.lr * m_new;
-    momentum[i] = (float)m_new;
-    params[i] = (float)th_new;
+    if (!h.adam) {
+      // SGD with momentum
+      const double m_new = h.beta * (double)momentum[i] + g;
+      const double th_new = (double)params[i] - h.lr * m_new;
+      momentum[i] = (float)m_new;
+      params[i] = (float)th_new;
+    } else {
+      // Adam with bias correction
+      const double m_new = h.beta * (double)momentum[i] + (1.0 - h.beta) * g;
+      const double v_new = h.beta2 * (double)second[i] + (1.0 - h.beta2) * g * g;
+      const double m_hat = m_new / (1.0 - std::pow(h.beta, (double)h.t));
+      const double v_hat = v_new / (1.0 - std::pow(h.beta2, (double)h.t));
+      const double den = std::sqrt(v_hat) + h.eps;
+      const double th_new = (double)params[i] - h.lr * m_hat / den;
+      const double g_hat = g / den;
+      out.su.add(g_hat);
+      out.su2.add(g_hat * g_hat);
+      momentum[i] = (float)m_new;
+      second[i] = (float)v_new;
+      params[i] = (float)th_new;
+    }
     prev_agg[i] = (float)g;
   }
 }
@@ -182,17 +206,31 @@ int dmxo_begin(dmxo* h, const int32_t* batch_sizes, float lr, float beta) {
   h->q.assign(h->K, Sum());
   h->V.assign(h->S, Sum());
   h->N.assign(h->S, Sum());
-  h->c = Sum(); h->pp = Sum();
+  h->c = Sum(); h->pp = Sum(); h->su = Sum(); h->su2 = Sum();
+  h->adam = false;
   h->next = 0;
   h->open = true;
   return kOk;
 }
 
+int dmxo_begin_adam(dmxo* h, const int32_t* batch_sizes, float lr, float beta1, float beta2, float eps, int64_t t) {
+  if (t < 1 || !(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps >= 0.f)) return kErrArg;
+  const int rc = dmxo_begin(h, batch_sizes, lr, beta1);
+  if (rc != kOk) return rc;
+  h->adam = true;
+  h->beta2 = (double)beta2;
+  h->eps = (double)eps;
+  h->t = t;
+  return kOk;
+}
+
 // Process elements [j0, j0+n). grads[k], params, momentum, prev_agg address element j0.
 // Ranges must arrive in ascending order without gaps, each starting on a multiple of 2^20.
-int dmxo_range(dmxo* h, int64_t j0, int64_t n, const void* const* grads, float* params,
-               float* momentum, float* prev_agg, int nthreads) {
+// `second` is Adam's second-moment array (element j0 first); null in SGD mode.
+int dmxo_range_adam(dmxo* h, int64_t j0, int64_t n, const void* const* grads, float* params,
+                    float* momentum, float* second, float* prev_agg, int nthreads) {
   if (!h || !h->open || !grads || !params || !momentum || !prev_agg) return kErrArg;
+  if (h->adam != (second != nullptr)) return kErrArg;
   if (j0 != h->next || j0 % kBlock != 0 || n < 1 || j0 + n > h->P) return kErrOrder;
   const int64_t nblocks = (n + kBlock - 1) / kBlock;
   std::vector<Partial> parts(nblocks);
@@ -201,7 +239,7 @@ int dmxo_range(dmxo* h, int64_t j0, int64_t n, const void* const* grads, float* 
   auto work = [&](int t) {
     for (int64_t blk = t; blk < nblocks; blk += nthreads) {
       int64_t a = j0 + blk * kBlock, e = a + kBlock < j0 + n ? a + kBlock : j0 + n;
-      run_block(*h, j0, a, e, grads, params, momentum, prev_agg, parts[blk]);
+      run_block(*h, j0, a, e, grads, params, momentum, second, prev_agg, parts[blk]);
     }
   };
   if (nthreads == 1) {
@@ -216,6 +254,8 @@ int dmxo_range(dmxo* h, int64_t j0, int64_t n, const void* const* grads, float* 
     for (int k = 0; k < h->K; ++k) h->q[k].add(p.q[k].value());
     h->c.add(p.c.value());
     h->pp.add(p.pp.value());
+    h->su.add(p.su.value());
+    h->su2.add(p.su2.value());
     for (size_t i = 0; i < p.V.size(); ++i) {
       h->V[p.seg_first + i].add(p.V[i].value());
       h->N[p.seg_first + i].add(p.N[i].value());
@@ -223,6 +263,11 @@ int dmxo_range(dmxo* h, int64_t j0, int64_t n, const void* const* grads, float* 
   }
   h->next = j0 + n;
   return kOk;
+}
+
+int dmxo_range(dmxo* h, int64_t j0, int64_t n, const void* const* grads, float* params,
+               float* momentum, float* prev_agg, int nthreads) {
+  return dmxo_range_adam(h, j0, n, grads, params, momentum, nullptr, prev_agg, nthreads);
 }
 
 int dmxo_end(dmxo* h, float* out_state) {
@@ -262,6 +307,13 @@ int dmxo_end(dmxo* h, float* out_state) {
   out_state[iSig] = (float)sig;
   out_state[iWq] = (float)(Qw.value() / B);
   out_state[iFlags] = (float)flags;
+  if (h->adam) {
+    const double mean = h->su.value() / (double)h->P;
+    const double var = h->su2.value() / (double)h->P - mean * mean;
+    out_state[12] = (float)mean;
+    out_state[13] = (float)var;
+    out_state[14] = (float)std::sqrt(var > 0.0 ? var : 0.0);
+  }
   for (int k = 0; k < K; ++k) out_state[iHdr + k] = (float)h->q[k].value();
   for (int s = 0; s < S; ++s) {
     out_state[iHdr + K + s] = K >= 2 ? (float)(h->V[s].value() / (K - 1)) : 0.0f;
@@ -278,6 +330,16 @@ int dmxo_step(dmxo* h, const void* const* grads, const int32_t* batch_sizes, flo
   int rc = dmxo_begin(h, batch_sizes, lr, beta);
   if (rc != kOk) return rc;
   rc = dmxo_range(h, 0, h->P, grads, params, momentum, prev_agg, nthreads);
+  if (rc != kOk) return rc;
+  return dmxo_end(h, out_state);
+}
+
+int dmxo_step_adam(dmxo* h, const void* const* grads, const int32_t* batch_sizes, float* params,
+                   float* momentum, float* second, float lr, float beta1, float beta2, float eps, int64_t t,
+                   float* prev_agg, float* out_state, int nthreads) {
+  int rc = dmxo_begin_adam(h, batch_sizes, lr, beta1, beta2, eps, t);
+  if (rc != kOk) return rc;
+  rc = dmxo_range_adam(h, 0, h->P, grads, params, momentum, second, prev_agg, nthreads);
   if (rc != kOk) return rc;
   return dmxo_end(h, out_state);
 }

@@ -51,8 +51,11 @@ def lib():
         L.dmxo_end.argtypes = [vp, vp]
         L.dmxo_step.argtypes = [vp, vp, vp, vp, vp, f32, f32, vp, vp, i32]
         L.dmxo_destroy.argtypes = [vp]
+        L.dmxo_begin_adam.argtypes = [vp, vp, f32, f32, f32, f32, i64]
+        L.dmxo_range_adam.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp, i32]
+        L.dmxo_step_adam.argtypes = [vp, vp, vp, vp, vp, vp, f32, f32, f32, f32, i64, vp, vp, i32]
         for f in (L.dmxo_create, L.dmxo_state_len, L.dmxo_begin, L.dmxo_range, L.dmxo_end,
-                  L.dmxo_step, L.dmxo_destroy):
+                  L.dmxo_step, L.dmxo_destroy, L.dmxo_begin_adam, L.dmxo_range_adam, L.dmxo_step_adam):
             f.restype = i32
         _lib = L
     return _lib
@@ -116,6 +119,35 @@ class Oracle:
         if rc != 0:
             raise OracleError(rc)
         return out
+
+    def step_adam(self, grads, batch_sizes, params, first, second, lr, beta1, beta2, eps, t, prev_agg, nthreads=1):
+        """Whole Adam step (t = 1-based step count) on full-length host arrays; returns out_state."""
+        gp = self._check_grads(grads, self.P)
+        self._check_state(self.P, params, first, second, prev_agg)
+        b = np.ascontiguousarray(batch_sizes, dtype=np.int32)
+        assert b.shape == (self.K,)
+        out = np.empty(self.state_len, dtype=np.float32)
+        rc = lib().dmxo_step_adam(self._h, gp, _ptr(b), _ptr(params), _ptr(first), _ptr(second), lr, beta1, beta2, eps,
+                                  int(t), _ptr(prev_agg), _ptr(out), int(nthreads))
+        if rc != 0:
+            raise OracleError(rc)
+        return out
+
+    def begin_adam(self, batch_sizes, lr, beta1, beta2, eps, t):
+        b = np.ascontiguousarray(batch_sizes, dtype=np.int32)
+        assert b.shape == (self.K,)
+        rc = lib().dmxo_begin_adam(self._h, _ptr(b), lr, beta1, beta2, eps, int(t))
+        if rc != 0:
+            raise OracleError(rc)
+
+    def range_adam(self, j0, grads, params, first, second, prev_agg, nthreads=1):
+        n = len(params)
+        gp = self._check_grads(grads, n)
+        self._check_state(n, params, first, second, prev_agg)
+        rc = lib().dmxo_range_adam(self._h, int(j0), n, gp, _ptr(params), _ptr(first), _ptr(second), _ptr(prev_agg),
+                                   int(nthreads))
+        if rc != 0:
+            raise OracleError(rc)
 
     # streaming form, for problems whose gradients do not fit in host memory at once
     def begin(self, batch_sizes, lr, beta):

@@ -19,7 +19,7 @@ ST_SIGMA2_NORM, ST_SIGMA_NORM, ST_WMEAN_SQNORM, ST_FLAGS = 8, 9, 10, 11
 ST_HDR = 16
 FLAG_NONFINITE, FLAG_G2_NONPOS, FLAG_COS_UNDEF, FLAG_SINGLE, FLAG_INTERNAL = 1, 2, 4, 8, 16
 
-EXPORTS = ("dmx_create", "dmx_state_len", "dmx_step", "dmx_step_host", "dmx_step_static", "dmx_set_profiling", "dmx_get_profile",
+EXPORTS = ("dmx_create", "dmx_state_len", "dmx_step", "dmx_step_adam", "dmx_step_host", "dmx_step_static", "dmx_set_profiling", "dmx_get_profile",
            "dmx_launches_per_step", "dmx_destroy", "dmx_strerror", "dmx_last_cuda_error")
 
 _lib = None
@@ -48,6 +48,8 @@ def lib():
         L.dmx_step.restype = i32
         L.dmx_step_host.argtypes = [vp, vp, vp, vp, vp, vp, f32, f32, vp, vp, vp, vp]
         L.dmx_step_host.restype = i32
+        L.dmx_step_adam.argtypes = [vp, vp, vp, vp, vp, vp, f32, f32, f32, f32, i64, vp, vp, vp]
+        L.dmx_step_adam.restype = i32
         L.dmx_step_static.argtypes = [i32, i64, vp, i32, i32, vp, vp, vp, vp, f32, f32, vp, vp, vp]
         L.dmx_step_static.restype = i32
         L.dmx_set_profiling.argtypes = [vp, i32]
@@ -102,6 +104,17 @@ def dmx_step_host(h, host_grad_ptrs, staging_ptrs, batch_sizes, params, momentum
     bs = (ctypes.c_int32 * K)(*[int(b) for b in batch_sizes])
     return lib().dmx_step_host(h, hp, sp, bs, int(params), int(momentum), float(lr), float(beta), int(prev_agg),
                                int(out_state_dev), int(out_state_host), int(stream) if stream else None)
+
+
+def dmx_step_adam(h, grad_ptrs, batch_sizes, params, first_moment, second_moment, lr, beta1, beta2, eps, t, prev_agg,
+                  out_state, stream=0) -> int:
+    """The step with the Adam update; t is the 1-based step count. Raw device addresses as dmx_step."""
+    K = len(grad_ptrs)
+    gp = (ctypes.c_void_p * K)(*[int(p) for p in grad_ptrs])
+    bs = (ctypes.c_int32 * K)(*[int(b) for b in batch_sizes])
+    return lib().dmx_step_adam(h, gp, bs, int(params), int(first_moment), int(second_moment), float(lr), float(beta1),
+                               float(beta2), float(eps), int(t), int(prev_agg), int(out_state),
+                               int(stream) if stream else None)
 
 
 def dmx_step_static(K, P, seg_offsets, grad_dtype, grad_ptrs, batch_sizes, params, momentum, lr, beta, prev_agg,
@@ -174,6 +187,29 @@ class Dmx:
                       lr, beta, prev_agg.data_ptr(), out_state.data_ptr(), stream)
         if rc != OK:
             raise DmxError(rc, "dmx_step")
+        return out_state
+
+    def step_adam(self, grads, batch_sizes, params, first_moment, second_moment, lr, beta1, beta2, eps, t, prev_agg,
+                  out_state=None, stream=None):
+        torch = self._torch
+        want = torch.float32 if self.dtype == F32 else torch.bfloat16
+        if len(grads) != self.K or len(batch_sizes) != self.K:
+            raise DmxError(ERR_ARG, "dmx_step_adam")
+        for g in grads:
+            if g.dtype != want or not g.is_cuda or not g.is_contiguous() or g.numel() != self.P:
+                raise DmxError(ERR_ARG, "dmx_step_adam (gradient tensor)")
+        for x in (params, first_moment, second_moment, prev_agg):
+            if x.dtype != torch.float32 or not x.is_cuda or not x.is_contiguous() or x.numel() != self.P:
+                raise DmxError(ERR_ARG, "dmx_step_adam (state tensor)")
+        if out_state is None:
+            out_state = torch.empty(self.state_len, dtype=torch.float32, device=params.device)
+        if stream is None:
+            stream = torch.cuda.current_stream(params.device).cuda_stream
+        rc = dmx_step_adam(self._h, [g.data_ptr() for g in grads], batch_sizes, params.data_ptr(),
+                           first_moment.data_ptr(), second_moment.data_ptr(), lr, beta1, beta2, eps, t,
+                           prev_agg.data_ptr(), out_state.data_ptr(), stream)
+        if rc != OK:
+            raise DmxError(rc, "dmx_step_adam")
         return out_state
 
     def step_host(self, host_grads, staging, batch_sizes, params, momentum, lr, beta, prev_agg, out_state_dev,

@@ -3,6 +3,7 @@
 #include "dmx.h"
 
 #include <algorithm>
+#include <cmath>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -26,10 +27,11 @@ constexpr uint64_t kMagic = 0x444d585f48414e44ull;  // "DMX_HAND"
 typedef void (*StepKernel)(const dmx::StepArgs);
 
 struct Plan {
-  StepKernel kernel = nullptr;
+  StepKernel kernel = nullptr;       // SGD-momentum update
+  StepKernel kernel_adam = nullptr;  // Adam update (one more state stream)
   int threads = 0;       // threads per CTA
   int tile = 0;          // elements per tile
-  size_t smem = 0;       // dynamic shared memory
+  size_t smem = 0, smem_adam = 0;    // dynamic shared memory
   int grid = 0;
 };
 
@@ -79,7 +81,8 @@ Plan direct_plan() {
   constexpr int NW = 8;
   constexpr int U = BF16 ? 4 : 8;
   Plan p;
-  p.kernel = dmx::direct_kernel<KT, BF16, NW, U>;
+  p.kernel = dmx::direct_kernel<KT, BF16, NW, U, false>;
+  p.kernel_adam = dmx::direct_kernel<KT, BF16, NW, U, true>;
   p.threads = NW * 32;
   p.tile = NW * 32 * dmx::Elem<BF16>::VEC;
   p.smem = 0;
@@ -101,12 +104,16 @@ Plan pick_direct(int K) {
 // 2-3 % slower on B200).
 template <int KT, bool BF16>
 Plan pipe_plan() {
-  typedef dmx::PipeCfg<KT, BF16, 8, 4, BF16 ? 11 : 12, 1> C;
+  typedef dmx::PipeCfg<KT, BF16, 8, 4, BF16 ? 11 : 12, 1, false> C;
+  typedef dmx::PipeCfg<KT, BF16, 8, 4, BF16 ? 11 : 12, 1, true> CA;
+  static_assert(C::T == CA::T && C::THREADS == CA::THREADS, "both updates share the tile tables");
   Plan p;
   p.kernel = dmx::pipe_kernel<C>;
+  p.kernel_adam = dmx::pipe_kernel<CA>;
   p.threads = C::THREADS;
   p.tile = C::T;
   p.smem = C::SMEM;
+  p.smem_adam = CA::SMEM;
   return p;
 }
 
@@ -166,8 +173,10 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   const bool direct = kv && std::strcmp(kv, "direct") == 0;
   Plan plan = direct ? (grad_dtype == DMX_BF16 ? pick_direct<true>(K) : pick_direct<false>(K))
                      : (grad_dtype == DMX_BF16 ? pick_pipe<true>(K) : pick_pipe<false>(K));
-  if (plan.smem > 48 * 1024 &&
-      !cuda_ok(cudaFuncSetAttribute(plan.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem))) {
+  if ((plan.smem > 48 * 1024 &&
+       !cuda_ok(cudaFuncSetAttribute(plan.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem))) ||
+      (plan.smem_adam > 48 * 1024 &&
+       !cuda_ok(cudaFuncSetAttribute(plan.kernel_adam, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_adam)))) {
     free_handle(h);
     return DMX_ERR_CUDA;
   }
@@ -262,9 +271,9 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
             upload(chunk_slot0, &h->chunk_slot0) && upload(seg_slots, &h->seg_slots) && upload(unit_lo, &h->unit_lo) &&
             upload(unit_hi, &h->unit_hi) && upload(seg_unit_ptr, &h->seg_unit_ptr);
   ok = ok && cuda_ok(cudaMalloc((void**)&h->segpart, (size_t)std::max(h->nunits, 1) * sizeof(double2)));
-  ok = ok && cuda_ok(cudaMalloc((void**)&h->rows, (size_t)nchunks * (K + 2) * sizeof(float)));
+  ok = ok && cuda_ok(cudaMalloc((void**)&h->rows, (size_t)nchunks * (K + 4) * sizeof(float)));
   ok = ok && cuda_ok(cudaMalloc((void**)&h->slots, (size_t)std::max<int64_t>(nslots, 1) * sizeof(float2)));
-  ok = ok && cuda_ok(cudaMalloc((void**)&h->colsum, (size_t)(K + 2) * sizeof(double)));
+  ok = ok && cuda_ok(cudaMalloc((void**)&h->colsum, (size_t)(K + 4) * sizeof(double)));
   ok = ok && cuda_ok(cudaMalloc((void**)&h->flags, 2 * sizeof(unsigned)));
   ok = ok && cuda_ok(cudaMemset(h->flags, 0, 2 * sizeof(unsigned)));
   ok = ok && cuda_ok(cudaDeviceSynchronize());
@@ -282,10 +291,21 @@ int dmx_state_len(const dmx_handle* h) {
   return DMX_ST_HDR + h->K + 2 * h->S;
 }
 
-int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes, float* params,
-             float* momentum, float lr, float beta, float* prev_agg, float* out_state, void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+
+struct AdamParams { float* second; float beta2, eps; int64_t t; };
+
+// One step with either update; `ap` is null for SGD with momentum.
+int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes, float* params,
+              float* momentum, float lr, float beta, float* prev_agg, float* out_state, void* cuda_stream,
+              const AdamParams* ap) {
   if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
   if (!grad_ptrs || !batch_sizes || !params || !momentum || !prev_agg || !out_state) return DMX_ERR_ARG;
+  if (ap && (!ap->second || ap->t < 1 || !(beta >= 0.f && beta < 1.f) || !(ap->beta2 >= 0.f && ap->beta2 < 1.f) ||
+             !(ap->eps >= 0.f)))
+    return DMX_ERR_ARG;
   const int K = h->K;
   const size_t esz = h->dtype == DMX_BF16 ? 2 : 4;
   const size_t gbytes = (size_t)h->P * esz, sbytes = (size_t)h->P * 4;
@@ -302,10 +322,12 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
     if ((uintptr_t)grad_ptrs[k] & 15) return DMX_ERR_ALIGN;
   if (((uintptr_t)params & 15) || ((uintptr_t)momentum & 15) || ((uintptr_t)prev_agg & 15) || ((uintptr_t)out_state & 3))
     return DMX_ERR_ALIGN;
-  const void* st[4] = {params, momentum, prev_agg, out_state};
-  const size_t sn[4] = {sbytes, sbytes, sbytes, obytes};
-  for (int i = 0; i < 4; ++i) {
-    for (int j = i + 1; j < 4; ++j)
+  if (ap && ((uintptr_t)ap->second & 15)) return DMX_ERR_ALIGN;
+  const void* st[5] = {params, momentum, prev_agg, out_state, ap ? ap->second : nullptr};
+  const size_t sn[5] = {sbytes, sbytes, sbytes, obytes, sbytes};
+  const int nst = ap ? 5 : 4;
+  for (int i = 0; i < nst; ++i) {
+    for (int j = i + 1; j < nst; ++j)
       if (overlap(st[i], sn[i], st[j], sn[j])) return DMX_ERR_ARG;
     for (int k = 0; k < K; ++k)
       if (overlap(st[i], sn[i], grad_ptrs[k], gbytes)) return DMX_ERR_ARG;
@@ -330,6 +352,13 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
   }
   A.params = params; A.momentum = momentum; A.prev = prev_agg;
   A.lr = lr; A.beta = beta; A.Bf = (float)B;
+  if (ap) {
+    // bias corrections in fp64 from the fp32 coefficients, handed over as fp32 factors
+    A.second = ap->second; A.beta2 = ap->beta2; A.eps = ap->eps;
+    A.omb1 = (float)(1.0 - (double)beta); A.omb2 = (float)(1.0 - (double)ap->beta2);
+    A.c1 = (float)(1.0 / (1.0 - std::pow((double)beta, (double)ap->t)));
+    A.c2 = (float)(1.0 / (1.0 - std::pow((double)ap->beta2, (double)ap->t)));
+  }
   A.K = K; A.S = h->S; A.P = h->P;
   A.tile_group = h->tile_group; A.group_stride = h->tile_group * h->plan.grid; A.nchunks = h->nchunks;
   A.seg_off = h->seg_off; A.tile_seg = h->tile_seg; A.cta_chunk0 = h->cta_chunk0; A.chunk_tile0 = h->chunk_tile0;
@@ -337,6 +366,7 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
   A.rows = h->rows; A.slots = h->slots; A.err = h->flags + 1;
 
   F.K = K; F.S = h->S; F.nchunks = h->nchunks; F.B = (double)B;
+  F.adam = ap ? 1 : 0; F.P = (double)h->P;
   F.rows = h->rows; F.slots = h->slots; F.seg_slots = h->seg_slots; F.nunits = h->nunits;
   F.unit_lo = h->unit_lo; F.unit_hi = h->unit_hi; F.seg_unit_ptr = h->seg_unit_ptr; F.segpart = h->segpart;
   F.colsum = h->colsum; F.ticket = h->flags; F.err = h->flags + 1; F.out_state = out_state;
@@ -344,10 +374,11 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const bool prof = h->profiling;
   if (prof && !cuda_ok(cudaEventRecord(h->ev[0], stream))) return DMX_ERR_CUDA;
-  h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A);
+  if (ap) h->plan.kernel_adam<<<h->plan.grid, h->plan.threads, h->plan.smem_adam, stream>>>(A);
+  else h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A);
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
   if (prof && !cuda_ok(cudaEventRecord(h->ev[1], stream))) return DMX_ERR_CUDA;
-  const int funits = K + 2 + h->nunits;   // one warp per chunk-row column and per segment unit
+  const int funits = K + 2 + 2 * F.adam + h->nunits;   // one warp per chunk-row column and per segment unit
   const int fblocks = (funits + dmx::kFinalWarps - 1) / dmx::kFinalWarps;
   dmx::finalize_kernel<<<fblocks, dmx::kFinalWarps * 32, 0, stream>>>(F);
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
@@ -356,6 +387,22 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
     h->profiled = true;
   }
   return DMX_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes, float* params,
+             float* momentum, float lr, float beta, float* prev_agg, float* out_state, void* cuda_stream) {
+  return step_impl(h, grad_ptrs, batch_sizes, params, momentum, lr, beta, prev_agg, out_state, cuda_stream, nullptr);
+}
+
+int dmx_step_adam(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes, float* params,
+                  float* first_moment, float* second_moment, float lr, float beta1, float beta2, float eps,
+                  int64_t t, float* prev_agg, float* out_state, void* cuda_stream) {
+  const AdamParams ap = {second_moment, beta2, eps, t};
+  return step_impl(h, grad_ptrs, batch_sizes, params, first_moment, lr, beta1, prev_agg, out_state, cuda_stream, &ap);
 }
 
 int dmx_step_host(dmx_handle* h, const void* const* host_grad_ptrs, void* const* staging_ptrs,

@@ -4,7 +4,9 @@
 //   g_j  = sum_k w_k x_kj                       (batch-size-weighted aggregate, w_k = b_k/B)
 //   d_j  = sum_k b_k (x_kj - g_j)^2             (spread of the workers around it)
 //   q_k += x_kj^2,  N_s += g_j^2,  V_s += d_j,  c += g_j a_j,  pp += a_j^2
-//   m_j  = beta m_j + g_j,  theta_j -= lr m_j,  a_j = g_j
+//   m_j  = beta m_j + g_j,  theta_j -= lr m_j,  a_j = g_j            (SGD with momentum), or
+//   m_j  = b1 m_j + (1-b1) g_j,  v_j = b2 v_j + (1-b2) g_j^2,
+//   theta_j -= lr mhat_j / (sqrt(vhat_j) + eps),  a_j = g_j            (Adam, bias-corrected)
 // The sums over k use the shifted one-pass form around a pivot worker (the one with the
 // largest batch): with e_k = x_k - x_pivot,  g = x_pivot + sum w_k e_k  and
 // d = sum b_k e_k^2 - B (sum w_k e_k)^2. Identical workers give d = 0 exactly, and the
@@ -39,7 +41,9 @@ struct StepArgs {
   float* params;
   float* momentum;
   float* prev;
-  float lr, beta, Bf;
+  float* second;         // Adam's second-moment estimate v (Adam kernels only)
+  float lr, beta, Bf;    // beta is the momentum coefficient, or Adam's beta1
+  float beta2, eps, omb1, omb2, c1, c2;   // Adam: beta2, eps, 1-beta1, 1-beta2, 1/(1-beta1^t), 1/(1-beta2^t)
   int K, S;
   int64_t P;
   int tile_group;              // R: tiles are dealt to the CTAs in groups of R consecutive tiles
@@ -52,13 +56,15 @@ struct StepArgs {
   const int32_t* chunk_tile0;  // nchunks: first tile of the chunk
   const int32_t* chunk_ntiles; // nchunks: tiles in the chunk (tile0, tile0+stride, ...)
   const int32_t* chunk_slot0;  // nchunks: first (V,N) slot of the chunk
-  float* rows;                 // (K+2) x nchunks, one column after the other: q_k..., c, pp
+  float* rows;                 // (K+4) x nchunks, one column after the other: q_k..., c, pp, and (Adam) su, su2
   float2* slots;               // nslots: (V partial, N partial), in the order the chunk emits them
   unsigned* err;               // set non-zero when a bounded wait gives up
 };
 
 struct FinalArgs {
   int K, S, nchunks, nunits;
+  int adam;                    // 1: also emit the optimizer-normalised statistics (columns K+2, K+3)
+  double P;
   int orig[kMaxK];             // processing slot -> caller's worker index
   double b[kMaxK];             // batch sizes, processing order
   double B;
@@ -69,7 +75,7 @@ struct FinalArgs {
   const int32_t* unit_hi;      //         at most kFinalPart slots long
   const int32_t* seg_unit_ptr; // S+1: units of segment s are [seg_unit_ptr[s], seg_unit_ptr[s+1])
   double2* segpart;            // nunits: (V, N) of each unit
-  double* colsum;              // K+2
+  double* colsum;              // K+4
   unsigned* ticket;
   unsigned* err;
   float* out_state;
@@ -137,11 +143,13 @@ struct Acc {
   u64 np[NP2], s1[NP2], s2[NP2];    // -pivot, sum w e, sum b e^2 (pairs)
   float q[KT];                      // per-worker sum of squares (chunk)
   float c, pp, vs, ns;              // <g,a>, |a|^2, current segment's V and N partials
+  float su, su2;                    // Adam only: sums of g/(sqrt(vhat)+eps) and of its square (chunk)
 
   __device__ __forceinline__ void reset_chunk() {
 #pragma unroll
     for (int k = 0; k < KT; ++k) q[k] = 0.f;
     c = pp = vs = ns = 0.f;
+    su = su2 = 0.f;
   }
   // k is a compile-time constant after unrolling at every call site, so q[k] is a register.
   __device__ __forceinline__ void add(int k, const u64* x, float w, float bf) {
@@ -180,7 +188,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 // Shared-memory work area of the reductions (used by the NW participating warps only).
 template <int KT, int NW>
 struct RedArea {
-  float rows[NW][KT + 2];
+  float rows[NW][KT + 4];
   float2 seg[kSegBuf][NW];
 };
 
@@ -254,15 +262,16 @@ __device__ __forceinline__ void segment_accumulate(Acc<KT, VEC>& a, const StepAr
 }
 
 // End of a chunk: last segment entry, drain, then q_k, c, pp -> the chunk's scratch row.
-template <int KT, int VEC, int NW>
+template <int KT, int VEC, int NW, bool ADAM = false>
 __device__ __forceinline__ void flush_chunk(Acc<KT, VEC>& a, const StepArgs& A, RedArea<KT, NW>* R, SegState& st,
                                             int chunk, float2* chunk_slots, int bar_id, int wid, int lane) {
   if (st.cur >= 0) seg_entry<KT, VEC, NW>(a, R, st, chunk_slots, bar_id, wid, lane);
-  constexpr int NV = KT + 2;
+  constexpr int NV = KT + 2 + (ADAM ? 2 : 0);
   float v[NV];
 #pragma unroll
   for (int k = 0; k < KT; ++k) v[k] = warp_sum(a.q[k]);
   v[KT] = warp_sum(a.c); v[KT + 1] = warp_sum(a.pp);
+  if constexpr (ADAM) { v[KT + 2] = warp_sum(a.su); v[KT + 3] = warp_sum(a.su2); }
   if (lane == 0) {
 #pragma unroll
     for (int i = 0; i < NV; ++i) R->rows[wid][i] = v[i];
@@ -282,9 +291,9 @@ __device__ __forceinline__ void flush_chunk(Acc<KT, VEC>& a, const StepArgs& A, 
 
 // Tile epilogue for one thread: aggregate, spread, update, statistics. State values
 // th/m/pv are inputs and are overwritten with the outputs (theta', m', g).
-template <int KT, int VEC>
+template <int KT, int VEC, bool ADAM = false>
 __device__ __forceinline__ void finish_elements(Acc<KT, VEC>& a, const StepArgs& A, float* th, float* m,
-                                                float* pv, float* dv, float* nv) {
+                                                float* pv, float* dv, float* nv, float* vv = nullptr) {
   float p[VEC], s1[VEC], s2[VEC];
 #pragma unroll
   for (int i = 0; i < VEC / 2; ++i) {
@@ -299,9 +308,21 @@ __device__ __forceinline__ void finish_elements(Acc<KT, VEC>& a, const StepArgs&
     nv[e] = g * g;
     a.c = fmaf(g, pv[e], a.c);
     a.pp = fmaf(pv[e], pv[e], a.pp);
-    const float mn = fmaf(A.beta, m[e], g);
-    th[e] = fmaf(-A.lr, mn, th[e]);
-    m[e] = mn;
+    if constexpr (ADAM) {
+      const float mn = fmaf(A.beta, m[e], A.omb1 * g);
+      const float vn = fmaf(A.beta2, vv[e], A.omb2 * (g * g));
+      const float den = __fsqrt_rn(vn * A.c2) + A.eps;
+      th[e] = fmaf(-A.lr, __fdiv_rn(mn * A.c1, den), th[e]);
+      const float gh = __fdiv_rn(g, den);          // the gradient in units of Adam's running scale
+      a.su += gh;
+      a.su2 = fmaf(gh, gh, a.su2);
+      m[e] = mn;
+      vv[e] = vn;
+    } else {
+      const float mn = fmaf(A.beta, m[e], g);
+      th[e] = fmaf(-A.lr, mn, th[e]);
+      m[e] = mn;
+    }
     pv[e] = g;
   }
 }
@@ -310,7 +331,7 @@ __device__ __forceinline__ void finish_elements(Acc<KT, VEC>& a, const StepArgs&
 // Direct tile: every thread streams its own 16-byte pieces with plain vector loads, U worker
 // loads in flight at a time. With GUARD it is the code path of the ragged last tile.
 
-template <int KT, bool BF16, bool GUARD, int U>
+template <int KT, bool BF16, bool GUARD, int U, bool ADAM = false>
 __device__ __forceinline__ void direct_tile(Acc<KT, Elem<BF16>::VEC>& a, const StepArgs& A, int64_t jt,
                                             float* dv, float* nv) {
   constexpr int VEC = Elem<BF16>::VEC;
@@ -347,12 +368,13 @@ __device__ __forceinline__ void direct_tile(Acc<KT, Elem<BF16>::VEC>& a, const S
     }
   }
   // state streams
-  float th[VEC], m[VEC], pv[VEC];
+  float th[VEC], m[VEC], pv[VEC], vv[ADAM ? VEC : 1];
   if constexpr (GUARD) {
 #pragma unroll
     for (int e = 0; e < VEC; ++e) {
       const bool ok = jt + e < A.P;
       th[e] = ok ? A.params[jt + e] : 0.f; m[e] = ok ? A.momentum[jt + e] : 0.f; pv[e] = ok ? A.prev[jt + e] : 0.f;
+      if constexpr (ADAM) vv[e] = ok ? A.second[jt + e] : 1.f;   // 1: keeps the unused lanes' divisions finite
     }
   } else {
 #pragma unroll
@@ -360,14 +382,18 @@ __device__ __forceinline__ void direct_tile(Acc<KT, Elem<BF16>::VEC>& a, const S
       uint4 r = ld_stream(A.params + jt + 4 * h);   unpack4f(r, th + 4 * h);
       r = ld_stream(A.momentum + jt + 4 * h);       unpack4f(r, m + 4 * h);
       r = ld_stream(A.prev + jt + 4 * h);           unpack4f(r, pv + 4 * h);
+      if constexpr (ADAM) { r = ld_stream(A.second + jt + 4 * h); unpack4f(r, vv + 4 * h); }
     }
   }
-  finish_elements<KT, VEC>(a, A, th, m, pv, dv, nv);
+  // (lanes beyond P carry g = 0 and v = 1: they add exact zeros to every sum)
+  finish_elements<KT, VEC, ADAM>(a, A, th, m, pv, dv, nv, vv);
   if constexpr (GUARD) {
 #pragma unroll
     for (int e = 0; e < VEC; ++e) {
-      if (jt + e < A.P) { A.params[jt + e] = th[e]; A.momentum[jt + e] = m[e]; A.prev[jt + e] = pv[e]; }
-      else { dv[e] = 0.f; nv[e] = 0.f; }
+      if (jt + e < A.P) {
+        A.params[jt + e] = th[e]; A.momentum[jt + e] = m[e]; A.prev[jt + e] = pv[e];
+        if constexpr (ADAM) A.second[jt + e] = vv[e];
+      } else { dv[e] = 0.f; nv[e] = 0.f; }
     }
   } else {
 #pragma unroll
@@ -375,17 +401,18 @@ __device__ __forceinline__ void direct_tile(Acc<KT, Elem<BF16>::VEC>& a, const S
       st_stream(A.params + jt + 4 * h, th[4 * h], th[4 * h + 1], th[4 * h + 2], th[4 * h + 3]);
       st_stream(A.momentum + jt + 4 * h, m[4 * h], m[4 * h + 1], m[4 * h + 2], m[4 * h + 3]);
       st_stream(A.prev + jt + 4 * h, pv[4 * h], pv[4 * h + 1], pv[4 * h + 2], pv[4 * h + 3]);
+      if constexpr (ADAM) st_stream(A.second + jt + 4 * h, vv[4 * h], vv[4 * h + 1], vv[4 * h + 2], vv[4 * h + 3]);
     }
   }
 }
 
 // The ragged last tile, kept out of line so that its registers do not weigh on the main loop.
-template <int KT, bool BF16>
+template <int KT, bool BF16, bool ADAM>
 __device__ __noinline__ void ragged_tile(Acc<KT, Elem<BF16>::VEC>& a, const StepArgs& A, int64_t jt, float* dv, float* nv) {
-  direct_tile<KT, BF16, true, 4>(a, A, jt, dv, nv);
+  direct_tile<KT, BF16, true, 4, ADAM>(a, A, jt, dv, nv);
 }
 
-template <int KT, bool BF16, int NW, int U>
+template <int KT, bool BF16, int NW, int U, bool ADAM>
 __global__ void __launch_bounds__(NW * 32)
 direct_kernel(const __grid_constant__ StepArgs A) {
   constexpr int VEC = Elem<BF16>::VEC;
@@ -407,14 +434,14 @@ direct_kernel(const __grid_constant__ StepArgs A) {
       int64_t tile_end = tile_begin + T;
       float dv[VEC], nv[VEC];
       if (tile_end <= A.P) {
-        direct_tile<KT, BF16, false, U>(a, A, jt, dv, nv);
+        direct_tile<KT, BF16, false, U, ADAM>(a, A, jt, dv, nv);
       } else {
         tile_end = A.P;
-        direct_tile<KT, BF16, true, U>(a, A, jt, dv, nv);
+        direct_tile<KT, BF16, true, U, ADAM>(a, A, jt, dv, nv);
       }
       segment_accumulate<KT, VEC, NW>(a, A, dv, nv, jt, tile_begin, tile_end, tseg, &R, st, chunk_slots, 1, wid, lane);
     }
-    flush_chunk<KT, VEC, NW>(a, A, &R, st, c, chunk_slots, 1, wid, lane);
+    flush_chunk<KT, VEC, NW, ADAM>(a, A, &R, st, c, chunk_slots, 1, wid, lane);
   }
 }
 
@@ -438,7 +465,8 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
   const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int K = F.K, S = F.S;
   const int unit = blockIdx.x * kFinalWarps + wid;
-  if (unit < K + 2) {
+  const int ncol = K + 2 + 2 * F.adam;
+  if (unit < ncol) {
     const float* col = F.rows + (int64_t)unit * F.nchunks;
     double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
     int c = lane;
@@ -448,8 +476,8 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
     for (; c < F.nchunks; c += 32) a0 += (double)col[c];
     const double acc = warp_sum_d((a0 + a1) + (a2 + a3));
     if (lane == 0) F.colsum[unit] = acc;
-  } else if (unit < K + 2 + F.nunits) {
-    const int u = unit - (K + 2);
+  } else if (unit < ncol + F.nunits) {
+    const int u = unit - ncol;
     const int lo = F.unit_lo[u], hi = F.unit_hi[u];
     double v = 0.0, n = 0.0, v1 = 0.0, n1 = 0.0, v2 = 0.0, n2 = 0.0, v3 = 0.0, n3 = 0.0;
     int i = lo + lane;
@@ -476,10 +504,10 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
   __threadfence();
   // last block: everything below reads what all blocks wrote. The K+2 column sums go through
   // shared memory so that the serial part at the end does not pay a global load per term.
-  __shared__ double cs[kMaxK + 2];
+  __shared__ double cs[kMaxK + 4];
   {
     const volatile double* gcs = F.colsum;
-    if (threadIdx.x < K + 2) cs[threadIdx.x] = gcs[threadIdx.x];
+    if (threadIdx.x < ncol) cs[threadIdx.x] = gcs[threadIdx.x];
   }
   const volatile double2* sp = F.segpart;
   float* out = F.out_state;
@@ -517,6 +545,13 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
     out[5] = (float)cosv; out[6] = (float)c; out[7] = (float)pp; out[8] = (float)sig2; out[9] = (float)sig;
     out[10] = (float)(Qw / B); out[11] = (float)flags;
     out[12] = out[13] = out[14] = out[15] = 0.f;
+    if (F.adam) {
+      // the gradient in units of Adam's running scale, ghat_j = g_j / (sqrt(vhat_j) + eps):
+      // its mean, variance and standard deviation across the parameters
+      const double mean = cs[K + 2] / F.P;
+      const double var = cs[K + 3] / F.P - mean * mean;
+      out[12] = (float)mean; out[13] = (float)var; out[14] = (float)sqrt(var > 0.0 ? var : 0.0);
+    }
     *F.ticket = 0u;
   }
 }
@@ -584,10 +619,11 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   return r;
 }
 
-template <int KT_, bool BF16_, int CW_, int G_, int NSTAGE_, int NSS_>
+template <int KT_, bool BF16_, int CW_, int G_, int NSTAGE_, int NSS_, bool ADAM_ = false>
 struct PipeCfg {
   static constexpr int KT = KT_, CW = CW_, G = G_, NSTAGE = NSTAGE_, NSS = NSS_;
-  static constexpr bool BF16 = BF16_;
+  static constexpr bool BF16 = BF16_, ADAM = ADAM_;
+  static constexpr int NST = ADAM ? 4 : 3;           // state streams: prev_agg, momentum, params (, second moment)
   static constexpr int VEC = Elem<BF16>::VEC;
   static constexpr int CT = CW * 32;                 // consumer threads
   static constexpr int THREADS = CT + 32;            // + the producer warp
@@ -595,7 +631,7 @@ struct PipeCfg {
   static constexpr int SLOT = CT * 16;               // one gradient stream's tile, bytes
   static constexpr int STAGE = G * SLOT;
   static constexpr int SSLOT = T * 4;                // one state stream's tile, bytes
-  static constexpr int SSTAGE = 3 * SSLOT;
+  static constexpr int SSTAGE = NST * SSLOT;
   static constexpr int RING = NSTAGE * STAGE;
   static constexpr int SRING = NSS * SSTAGE;
   static constexpr int RED = (int)((sizeof(RedArea<KT, CW>) + 15) / 16 * 16);
@@ -609,7 +645,7 @@ struct PipeCfg {
 template <class C>
 __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_constant__ StepArgs A) {
   constexpr int KT = C::KT, VEC = C::VEC, CW = C::CW, G = C::G, NSTAGE = C::NSTAGE, NSS = C::NSS, T = C::T;
-  constexpr bool BF16 = C::BF16;
+  constexpr bool BF16 = C::BF16, ADAM = C::ADAM;
   extern __shared__ __align__(128) unsigned char smem[];
   const uint32_t ring = smem_u32(smem);
   const uint32_t sring = ring + C::RING;
@@ -666,8 +702,8 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
         armed_s |= 1u << ss;
         par_s = (par_s & ~(1u << ss)) | (sphase << ss);
         __syncwarp();
-        if (lane < 3) {
-          const float* src = lane == 0 ? A.prev : (lane == 1 ? A.momentum : A.params);
+        if (lane < C::NST) {
+          const float* src = lane == 0 ? A.prev : (lane == 1 ? A.momentum : (lane == 2 ? A.params : A.second));
           bulk_load(sring + ss * C::SSTAGE + lane * C::SSLOT, src + tile_begin, C::SSLOT, full_s + 8 * ss, pol);
         }
         if (++ss == NSS) { ss = 0; sphase ^= 1u; }
@@ -728,7 +764,7 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
           }
         }
         ok = mbar_wait(full_s + 8 * ss, sphase, give_up, A.err) && ok;
-        float th[VEC], m[VEC], pv[VEC];
+        float th[VEC], m[VEC], pv[VEC], vv[ADAM ? VEC : 1];
         {
           const uint32_t src = sring + ss * C::SSTAGE + tid * (VEC * 4);
 #pragma unroll
@@ -736,18 +772,20 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
             uint4 r = lds128(src + 16 * h);               unpack4f(r, pv + 4 * h);
             r = lds128(src + C::SSLOT + 16 * h);          unpack4f(r, m + 4 * h);
             r = lds128(src + 2 * C::SSLOT + 16 * h);      unpack4f(r, th + 4 * h);
+            if constexpr (ADAM) { r = lds128(src + 3 * C::SSLOT + 16 * h); unpack4f(r, vv + 4 * h); }
           }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_s + 8 * ss);
         if (++ss == NSS) { ss = 0; sphase ^= 1u; }
-        finish_elements<KT, VEC>(a, A, th, m, pv, dv, nv);
+        finish_elements<KT, VEC, ADAM>(a, A, th, m, pv, dv, nv, vv);
         if (ok) {
 #pragma unroll
           for (int h = 0; h < VEC / 4; ++h) {
             st_stream(A.params + jt + 4 * h, th[4 * h], th[4 * h + 1], th[4 * h + 2], th[4 * h + 3]);
             st_stream(A.momentum + jt + 4 * h, m[4 * h], m[4 * h + 1], m[4 * h + 2], m[4 * h + 3]);
             st_stream(A.prev + jt + 4 * h, pv[4 * h], pv[4 * h + 1], pv[4 * h + 2], pv[4 * h + 3]);
+            if constexpr (ADAM) st_stream(A.second + jt + 4 * h, vv[4 * h], vv[4 * h + 1], vv[4 * h + 2], vv[4 * h + 3]);
           }
         }
       } else {
@@ -755,14 +793,14 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
         // through copies, so that only the copies (not the loop's registers) have their address taken
         Acc<KT, VEC> a2 = a;
         float dv2[VEC], nv2[VEC];
-        ragged_tile<KT, BF16>(a2, A, jt, dv2, nv2);
+        ragged_tile<KT, BF16, ADAM>(a2, A, jt, dv2, nv2);
         a = a2;
 #pragma unroll
         for (int e = 0; e < VEC; ++e) { dv[e] = dv2[e]; nv[e] = nv2[e]; }
       }
       segment_accumulate<KT, VEC, CW>(a, A, dv, nv, jt, tile_begin, tile_end, tseg, R, st, chunk_slots, 1, wid, lane);
     }
-    flush_chunk<KT, VEC, CW>(a, A, R, st, c, chunk_slots, 1, wid, lane);
+    flush_chunk<KT, VEC, CW, ADAM>(a, A, R, st, c, chunk_slots, 1, wid, lane);
   }
 }
 

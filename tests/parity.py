@@ -29,6 +29,38 @@ def cond_vectors(grads_f32, b, params_in, momentum_in, lr, beta):
     return cg, cm, ct
 
 
+def cond_vectors_adam(grads_f32, b, params_in, m_in, v_in, lr, beta1, beta2, eps, t):
+    """Forward-error scales of g, m', v', theta' under the Adam update (float64 arrays)."""
+    w = np.asarray(b, np.float64) / float(np.sum(b))
+    cg = np.zeros(len(params_in), np.float64)
+    g = np.zeros(len(params_in), np.float64)
+    for k, x in enumerate(grads_f32):
+        cg += w[k] * np.abs(x.astype(np.float64))
+        g += w[k] * x.astype(np.float64)
+    b1, b2 = float(np.float32(beta1)), float(np.float32(beta2))
+    cm = np.abs(b1 * m_in.astype(np.float64)) + (1 - b1) * cg
+    cv = b2 * np.abs(v_in.astype(np.float64)) + (1 - b2) * 2 * cg * cg
+    c1, c2 = 1 / (1 - b1 ** t), 1 / (1 - b2 ** t)
+    m_new = b1 * m_in.astype(np.float64) + (1 - b1) * g
+    v_new = b2 * v_in.astype(np.float64) + (1 - b2) * g * g
+    root = np.sqrt(v_new * c2)
+    den = root + float(np.float32(eps))
+    u = m_new * c1 / np.maximum(den, 1e-300)
+    cu = c1 * cm / np.maximum(den, 1e-300) + np.abs(u) * c2 * cv / np.maximum(2 * root * den, 1e-300)
+    ct = np.abs(params_in.astype(np.float64)) + abs(float(np.float32(lr))) * (np.abs(u) + cu)
+    return cg, cm, cv, ct
+
+
+def check_vectors_adam(dtype, gpu_vecs, ref_vecs, conds, what=""):
+    tol = TOL_V[dtype]
+    errs = {}
+    for name, g, r, c in zip(("agg", "first_moment", "second_moment", "params"), gpu_vecs, ref_vecs, conds):
+        e = vec_err(g, r, c)
+        errs[name] = e
+        assert e <= tol, "%s %s: max scaled error %.3e > %.1e" % (what, name, e, tol)
+    return errs
+
+
 def vec_err(gpu, ref, cond):
     """max over elements of |gpu-ref| / max(|ref|, cond) (0/0 counts as 0)."""
     gpu = gpu.astype(np.float64); ref = ref.astype(np.float64)
@@ -56,7 +88,7 @@ def seg_scales(cg, seg, lo=0):
     return cs[idx[1:]] - cs[idx[:-1]]
 
 
-def check_state(gpu, ref, K, S, seg, b, what="", tol=TOL_S, seg_scale=None):
+def check_state(gpu, ref, K, S, seg, b, what="", tol=TOL_S, seg_scale=None, adam=False):
     """Compare two out_state vectors (float32 arrays). Returns the max relative error seen.
 
     seg_scale[s] = sum_{j in s} cond_j^2: a segment of a few elements inherits the forward
@@ -107,7 +139,16 @@ def check_state(gpu, ref, K, S, seg, b, what="", tol=TOL_S, seg_scale=None):
     if abs(G2) > tol * max(A, 1e-300):
         mask |= 2
     assert (fg & mask) == (fr & mask), "%s flags gpu %d ref %d" % (what, fg, fr)
-    assert np.all(gpu[12:16] == 0)
+    if adam:
+        # mean, variance, std of ghat = g/(sqrt(vhat)+eps) over the parameters: judged against its rms
+        rms2 = ref[13] + ref[12] ** 2
+        assert abs(gpu[12] - ref[12]) <= tol * np.sqrt(rms2), "%s ghat mean gpu %.9g ref %.9g" % (what, gpu[12], ref[12])
+        assert abs(gpu[13] - ref[13]) <= 2 * tol * rms2, "%s ghat var gpu %.9g ref %.9g" % (what, gpu[13], ref[13])
+        if ref[13] > 1e-3 * rms2:
+            assert abs(gpu[14] - ref[14]) <= 2 * tol * np.sqrt(rms2), "%s ghat std gpu %.9g ref %.9g" % (what, gpu[14], ref[14])
+        assert gpu[15] == 0
+    else:
+        assert np.all(gpu[12:16] == 0)
     for k in range(K):
         rel(HDR + k, "worker_sqnorm[%d]" % k)
     for s in range(S):

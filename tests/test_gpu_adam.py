@@ -1,0 +1,88 @@
+"""Parity of dmx_step_adam (through the C ABI) with the oracle's Adam mode. Needs a GPU."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle.dmx_oracle import Oracle
+from paper_2510_08522_b200 import workload as W
+from tests import parity as PT
+
+pytestmark = pytest.mark.gpu
+NTHREADS = max(1, min(32, os.cpu_count() or 1))
+LR, B1, B2, EPS = 1e-3, 0.9, 0.999, 1e-8
+
+
+def _torch():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    return torch
+
+
+def lock_step_adam(wl, steps, v0=0.0):
+    torch = _torch()
+    import paper_2510_08522_b200 as D
+    dp = W.DeviceProblem(wl)
+    second = torch.full((wl.P,), v0, dtype=torch.float32, device="cuda")
+    orc = Oracle(wl.K, wl.P, dp.seg, wl.dtype)
+    d = D.Dmx(wl.K, wl.P, dp.seg, wl.dtype)
+    worst = {}
+    for t in range(1, steps + 1):
+        # Lock step: the oracle starts every step from the CUDA path's state. Adam's update is
+        # sign-like where |g| is near eps, so an element whose aggregate cancels to ~0 takes a
+        # legitimately different step on the two sides (its forward-error scale says so) and a
+        # free-running comparison would carry that difference in theta for ever.
+        hp, hm, hv, ha = (x.cpu().numpy().copy() for x in (dp.params, dp.momentum, second, dp.prev_agg))
+        b = dp.fill()
+        raw, wide = PT.grads_to_host(torch, dp.grads, wl.dtype)
+        conds = PT.cond_vectors_adam(wide, b, hp, hm, hv, LR, B1, B2, EPS, t)
+        ref = orc.step_adam(raw, b, hp, hm, hv, LR, B1, B2, EPS, t, ha, nthreads=NTHREADS)
+        st = d.step_adam(dp.grads, b, dp.params, dp.momentum, second, LR, B1, B2, EPS, t, dp.prev_agg)
+        torch.cuda.synchronize()
+        what = "%s adam step %d" % (wl.name, t)
+        e = PT.check_vectors_adam(wl.dtype, tuple(x.cpu().numpy() for x in (dp.prev_agg, dp.momentum, second, dp.params)),
+                                  (ha, hm, hv, hp), conds, what)
+        e["state"] = PT.check_state(st.cpu().numpy(), ref, wl.K, wl.S, dp.seg, b, what,
+                                    seg_scale=PT.seg_scales(conds[0], dp.seg), adam=True)
+        for k, v in e.items():
+            worst[k] = max(worst.get(k, 0.0), v)
+        dp.advance()
+    d.close()
+    return worst
+
+
+@pytest.mark.parametrize("idx,P,steps", [(0, 262_147, 3), (1, 333_337, 8), (2, 401_239, 8), (3, 290_011, 4), (4, 523_777, 4)])
+def test_adam_scaled_workloads_multi_step(idx, P, steps):
+    print(lock_step_adam(W.WORKLOADS[idx].scaled(P=P, steps=steps), steps))
+
+
+def test_adam_cfg1_full_size():
+    wl = W.WORKLOADS[1]
+    print(lock_step_adam(wl.scaled(P=wl.P, steps=4), 4))
+
+
+@pytest.mark.parametrize("K,P", [(1, 5), (3, 1023), (5, 2049), (33, 20_011), (64, 9_973)])
+def test_adam_shapes(K, P):
+    wl = W.Workload("adam-K%d-P%d" % (K, P), K, P, 3, W.BF16 if K % 2 else W.F32, 2, 11, "equal", "fixed4", True)
+    print(lock_step_adam(wl, 2, v0=0.25))
+
+
+def test_adam_argument_errors():
+    torch = _torch()
+    from paper_2510_08522_b200 import binding as B
+    P = 4096
+    rc, h = B.dmx_create(2, P, [0, P], 0)
+    assert rc == 0
+    g = [torch.zeros(P, device="cuda") for _ in range(2)]
+    s = [torch.zeros(P + 8, device="cuda") for _ in range(4)]
+    out = torch.zeros(B.dmx_state_len(h), device="cuda")
+    call = lambda **kw: B.dmx_step_adam(h, [x.data_ptr() for x in g], [1, 2], s[0].data_ptr(), s[1].data_ptr(),
+                                        kw.get("v", s[2].data_ptr()), 1e-3, kw.get("b1", 0.9), kw.get("b2", 0.999),
+                                        kw.get("eps", 1e-8), kw.get("t", 1), s[3].data_ptr(), out.data_ptr())
+    assert call() == B.OK
+    assert call(t=0) == B.ERR_ARG and call(b1=1.0) == B.ERR_ARG and call(b2=-0.5) == B.ERR_ARG and call(eps=-1.0) == B.ERR_ARG
+    assert call(v=0) == B.ERR_ARG
+    assert call(v=s[2].data_ptr() + 4) == B.ERR_ALIGN
+    assert call(v=s[1].data_ptr()) == B.ERR_ARG          # second moment aliases the first
+    torch.cuda.synchronize()
+    assert B.dmx_destroy(h) == B.OK
