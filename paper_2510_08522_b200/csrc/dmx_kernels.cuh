@@ -108,6 +108,9 @@ __device__ __forceinline__ int tile_of(const StepArgs& A, int t0, int i) {
   return t0 + g * A.group_stride + (i - g * A.tile_group);
 }
 
+__device__ __forceinline__ float sqrt_approx(float x) { float r; asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+__device__ __forceinline__ float rcp_approx(float x) { float r; asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+
 template <bool BF16> struct Elem;
 template <> struct Elem<false> { static constexpr int VEC = 4; typedef float T; };
 template <> struct Elem<true>  { static constexpr int VEC = 8; typedef uint16_t T; };
@@ -291,29 +294,34 @@ __device__ __forceinline__ void flush_chunk(Acc<KT, VEC>& a, const StepArgs& A, 
 
 // Tile epilogue for one thread: aggregate, spread, update, statistics. State values
 // th/m/pv are inputs and are overwritten with the outputs (theta', m', g).
-template <int KT, int VEC, bool ADAM = false>
-__device__ __forceinline__ void finish_elements(Acc<KT, VEC>& a, const StepArgs& A, float* th, float* m,
-                                                float* pv, float* dv, float* nv, float* vv = nullptr) {
-  float p[VEC], s1[VEC], s2[VEC];
+// Four consecutive elements (pairs E0/2 and E0/2+1 of the thread) at a time, so that the
+// state values of only four elements are live at once.
+template <int KT, int VEC, bool ADAM, int E0>
+__device__ __forceinline__ void finish4(Acc<KT, VEC>& a, const StepArgs& A, float* th, float* m, float* pv,
+                                        float* dv, float* nv, float* vv) {
+  float p[4], s1[4], s2[4];
 #pragma unroll
-  for (int i = 0; i < VEC / 2; ++i) {
-    upk(a.np[i], p[2 * i], p[2 * i + 1]);
-    upk(a.s1[i], s1[2 * i], s1[2 * i + 1]);
-    upk(a.s2[i], s2[2 * i], s2[2 * i + 1]);
+  for (int i = 0; i < 2; ++i) {
+    upk(a.np[E0 / 2 + i], p[2 * i], p[2 * i + 1]);
+    upk(a.s1[E0 / 2 + i], s1[2 * i], s1[2 * i + 1]);
+    upk(a.s2[E0 / 2 + i], s2[2 * i], s2[2 * i + 1]);
   }
 #pragma unroll
-  for (int e = 0; e < VEC; ++e) {
+  for (int e = 0; e < 4; ++e) {
     const float g = s1[e] - p[e];                // p holds the negated pivot
-    dv[e] = fmaf(-A.Bf * s1[e], s1[e], s2[e]);
-    nv[e] = g * g;
+    dv[E0 + e] = fmaf(-A.Bf * s1[e], s1[e], s2[e]);
+    nv[E0 + e] = g * g;
     a.c = fmaf(g, pv[e], a.c);
     a.pp = fmaf(pv[e], pv[e], a.pp);
     if constexpr (ADAM) {
       const float mn = fmaf(A.beta, m[e], A.omb1 * g);
       const float vn = fmaf(A.beta2, vv[e], A.omb2 * (g * g));
-      const float den = __fsqrt_rn(vn * A.c2) + A.eps;
-      th[e] = fmaf(-A.lr, __fdiv_rn(mn * A.c1, den), th[e]);
-      const float gh = __fdiv_rn(g, den);          // the gradient in units of Adam's running scale
+      // one approximate square root and one approximate reciprocal per element (each within
+      // 2^-22 relative, subnormals kept): IEEE sqrt and two divisions made the bf16 consumer
+      // compute-bound
+      const float rden = rcp_approx(sqrt_approx(vn * A.c2) + A.eps);
+      th[e] = fmaf(-A.lr, (mn * A.c1) * rden, th[e]);
+      const float gh = g * rden;                   // the gradient in units of Adam's running scale
       a.su += gh;
       a.su2 = fmaf(gh, gh, a.su2);
       m[e] = mn;
@@ -325,6 +333,13 @@ __device__ __forceinline__ void finish_elements(Acc<KT, VEC>& a, const StepArgs&
     }
     pv[e] = g;
   }
+}
+
+template <int KT, int VEC, bool ADAM = false>
+__device__ __forceinline__ void finish_elements(Acc<KT, VEC>& a, const StepArgs& A, float* th, float* m,
+                                                float* pv, float* dv, float* nv, float* vv = nullptr) {
+  finish4<KT, VEC, ADAM, 0>(a, A, th, m, pv, dv, nv, vv);
+  if constexpr (VEC == 8) finish4<KT, VEC, ADAM, 4>(a, A, th + 4, m + 4, pv + 4, dv, nv, ADAM ? vv + 4 : vv);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -764,28 +779,28 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
           }
         }
         ok = mbar_wait(full_s + 8 * ss, sphase, give_up, A.err) && ok;
-        float th[VEC], m[VEC], pv[VEC], vv[ADAM ? VEC : 1];
-        {
-          const uint32_t src = sring + ss * C::SSTAGE + tid * (VEC * 4);
+        // the tile's state in halves of four elements: load, update, store (only one half's
+        // values are live at a time; the stage is released after the last load)
+        const uint32_t ssrc = sring + ss * C::SSTAGE + tid * (VEC * 4);
 #pragma unroll
-          for (int h = 0; h < VEC / 4; ++h) {
-            uint4 r = lds128(src + 16 * h);               unpack4f(r, pv + 4 * h);
-            r = lds128(src + C::SSLOT + 16 * h);          unpack4f(r, m + 4 * h);
-            r = lds128(src + 2 * C::SSLOT + 16 * h);      unpack4f(r, th + 4 * h);
-            if constexpr (ADAM) { r = lds128(src + 3 * C::SSLOT + 16 * h); unpack4f(r, vv + 4 * h); }
+        for (int h = 0; h < VEC / 4; ++h) {
+          float th[4], m[4], pv[4], vv[4];
+          uint4 r = lds128(ssrc + 16 * h);                  unpack4f(r, pv);
+          r = lds128(ssrc + C::SSLOT + 16 * h);             unpack4f(r, m);
+          r = lds128(ssrc + 2 * C::SSLOT + 16 * h);         unpack4f(r, th);
+          if constexpr (ADAM) { r = lds128(ssrc + 3 * C::SSLOT + 16 * h); unpack4f(r, vv); }
+          if (h == VEC / 4 - 1) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_s + 8 * ss);
+            if (++ss == NSS) { ss = 0; sphase ^= 1u; }
           }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty_s + 8 * ss);
-        if (++ss == NSS) { ss = 0; sphase ^= 1u; }
-        finish_elements<KT, VEC, ADAM>(a, A, th, m, pv, dv, nv, vv);
-        if (ok) {
-#pragma unroll
-          for (int h = 0; h < VEC / 4; ++h) {
-            st_stream(A.params + jt + 4 * h, th[4 * h], th[4 * h + 1], th[4 * h + 2], th[4 * h + 3]);
-            st_stream(A.momentum + jt + 4 * h, m[4 * h], m[4 * h + 1], m[4 * h + 2], m[4 * h + 3]);
-            st_stream(A.prev + jt + 4 * h, pv[4 * h], pv[4 * h + 1], pv[4 * h + 2], pv[4 * h + 3]);
-            if constexpr (ADAM) st_stream(A.second + jt + 4 * h, vv[4 * h], vv[4 * h + 1], vv[4 * h + 2], vv[4 * h + 3]);
+          if (h == 0) finish4<KT, VEC, ADAM, 0>(a, A, th, m, pv, dv, nv, vv);
+          else finish4<KT, VEC, ADAM, (VEC == 8 ? 4 : 0)>(a, A, th, m, pv, dv, nv, vv);
+          if (ok) {
+            st_stream(A.params + jt + 4 * h, th[0], th[1], th[2], th[3]);
+            st_stream(A.momentum + jt + 4 * h, m[0], m[1], m[2], m[3]);
+            st_stream(A.prev + jt + 4 * h, pv[0], pv[1], pv[2], pv[3]);
+            if constexpr (ADAM) st_stream(A.second + jt + 4 * h, vv[0], vv[1], vv[2], vv[3]);
           }
         }
       } else {

@@ -86,3 +86,35 @@ def test_adam_argument_errors():
     assert call(v=s[1].data_ptr()) == B.ERR_ARG          # second moment aliases the first
     torch.cuda.synchronize()
     assert B.dmx_destroy(h) == B.OK
+
+
+def test_adam_full_size_streamed_cfg4():
+    """One Adam step at the largest workload's full size, gradients streamed to the oracle in ranges."""
+    torch = _torch()
+    import paper_2510_08522_b200 as D
+    wl = W.WORKLOADS[4]
+    dp = W.DeviceProblem(wl)
+    orc = Oracle(wl.K, wl.P, dp.seg, wl.dtype)
+    d = D.Dmx(wl.K, wl.P, dp.seg, wl.dtype)
+    second = torch.full((wl.P,), 1e-3, dtype=torch.float32, device="cuda")
+    dp.momentum.normal_(0.0, 0.01)                      # a non-trivial first moment
+    b = dp.fill()
+    t = 5
+    ins = [x.clone() for x in (dp.params, dp.momentum, second, dp.prev_agg)]
+    st = d.step_adam(dp.grads, b, dp.params, dp.momentum, second, LR, B1, B2, EPS, t, dp.prev_agg)
+    torch.cuda.synchronize()
+    orc.begin_adam(b, LR, B1, B2, EPS, t)
+    scale = np.zeros(wl.S)
+    span = 4 << 20
+    for lo in range(0, wl.P, span):
+        hi = min(wl.P, lo + span)
+        raw, wide = PT.grads_to_host(torch, dp.grads, wl.dtype, lo, hi)
+        hp, hm, hv, ha = (x[lo:hi].cpu().numpy() for x in ins)
+        conds = PT.cond_vectors_adam(wide, b, hp, hm, hv, LR, B1, B2, EPS, t)
+        scale += PT.seg_scales(conds[0], dp.seg, lo)
+        orc.range_adam(lo, raw, hp, hm, hv, ha, nthreads=NTHREADS)
+        gpu = tuple(x[lo:hi].cpu().numpy() for x in (dp.prev_agg, dp.momentum, second, dp.params))
+        PT.check_vectors_adam(wl.dtype, gpu, (ha, hm, hv, hp), conds, "%s adam [%d,%d)" % (wl.name, lo, hi))
+    ref = orc.end()
+    PT.check_state(st.cpu().numpy(), ref, wl.K, wl.S, dp.seg, b, wl.name + " adam", seg_scale=scale, adam=True)
+    d.close()
