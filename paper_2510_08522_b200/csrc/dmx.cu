@@ -98,14 +98,15 @@ Plan pick_direct(int K) {
   return direct_plan<64, BF16>();
 }
 
-// Pipelined (bulk-copy ring) kernels. Ring geometry: 8 consumer warps, 4 gradient streams per
-// 16 KB stage (smaller stages lose to the per-stage synchronisation, larger ones leave too few
-// in flight); as many stages as fit beside one state stage (a second state stage measured
-// 2-3 % slower on B200).
+// Pipelined (bulk-copy ring) kernels. Ring geometry: 7 consumer warps + the producer warp = 8
+// warps, so that a thread may use up to 255 registers (9 warps are allocated as 12 and cap it
+// at 168, which spilled at K = 32); 4 gradient streams per 14 KB stage (smaller stages lose to
+// the per-stage synchronisation, larger ones leave too few in flight); as many stages as fit
+// beside one state stage (a second state stage measured 2-3 % slower on B200).
 template <int KT, bool BF16>
 Plan pipe_plan() {
-  typedef dmx::PipeCfg<KT, BF16, 8, 4, BF16 ? 11 : 12, 1, false> C;
-  typedef dmx::PipeCfg<KT, BF16, 8, 4, BF16 ? 11 : 12, 1, true> CA;
+  typedef dmx::PipeCfg<KT, BF16, 7, 4, BF16 ? 13 : 14, 1, false> C;
+  typedef dmx::PipeCfg<KT, BF16, 7, 4, BF16 ? 12 : 14, 1, true> CA;
   static_assert(C::T == CA::T && C::THREADS == CA::THREADS, "both updates share the tile tables");
   Plan p;
   p.kernel = dmx::pipe_kernel<C>;
@@ -192,7 +193,12 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   // g mod grid. A CTA's tiles are cut into chunks of about `DMX_CHUNK_TILES` tiles so that fp32
   // per-thread partials stay short. The cut is a function of (P, tile, grid, R) only, so
   // results are reproducible on a given device.
-  const int R = std::max(1, std::min(env_int("DMX_TILE_GROUP", 4), 1 << 16));   // tuning knob: tiles per group
+  // Groups of 4 tiles measured 0.5-1 % faster than single tiles on the large workloads, but a
+  // CTA's share is a whole number of groups: keep at least 64 groups per CTA so that the
+  // imbalance stays below ~1.5 % (small problems fall back to groups of 2 or 1).
+  const int64_t sm_ctas = (int64_t)prop.multiProcessorCount * occ;
+  const int auto_R = ntiles >= 4 * 64 * sm_ctas ? 4 : (ntiles >= 2 * 64 * sm_ctas ? 2 : 1);
+  const int R = std::max(1, std::min(env_int("DMX_TILE_GROUP", auto_R), 1 << 16));   // tuning knob: tiles per group
   const int chunk_groups = std::max(1, env_int("DMX_CHUNK_TILES", 32) / R);
   const int64_t ngroups = (ntiles + R - 1) / R;
   plan.grid = (int)std::min<int64_t>((int64_t)prop.multiProcessorCount * occ, ngroups);
