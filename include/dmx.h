@@ -189,6 +189,29 @@ int dmx_get_profile(dmx_handle* h, float* fused_ms, float* finalize_ms);
 int dmx_launches_per_step(const dmx_handle* h);
 
 /*
+ * Window statistics of the state vector over k consecutive steps, kept on the device.
+ * The controller acts on metrics aggregated over k iterations (Section "System architecture";
+ * Section "State representation": state vectors are built from metrics collected every k
+ * iterations, as means and standard deviations); with this the host reads one vector per
+ * window instead of one per step.
+ *   dmx_agg_create   state_len = dmx_state_len(h) (> DMX_ST_FLAGS), k >= 1; allocates two fp64
+ *                    vectors on the current device
+ *   dmx_agg_push     out_state: DEVICE, state_len fp32, as written by a step (enqueue the push on
+ *                    the step's stream, after it); window_out: DEVICE, 2*state_len fp32. On every
+ *                    k-th push window_out receives, per entry i over the window's k vectors,
+ *                    mean (at i) and population standard deviation sqrt(sum (x-mean)^2 / k) (at
+ *                    state_len + i), and the window restarts; entry DMX_ST_FLAGS gets the OR of
+ *                    the k flag words and spread 0. Other pushes leave window_out untouched.
+ *                    *emitted (HOST, may be NULL) is set to 1 on the pushes that write, else 0.
+ *                    Asynchronous, no allocation.
+ * Errors: DMX_ERR_ARG, DMX_ERR_NOMEM, DMX_ERR_HANDLE, DMX_ERR_CUDA.
+ */
+typedef struct dmx_agg dmx_agg;
+int dmx_agg_create(int state_len, int k, dmx_agg** out);
+int dmx_agg_push(dmx_agg* a, const float* out_state, float* window_out, int* emitted, void* cuda_stream);
+int dmx_agg_destroy(dmx_agg* a);
+
+/*
  * dmx_step_static — the same step without a handle and without any allocation.
  * (The paper has no counterpart: this entry point exists for the library's callers only.)
  *

@@ -344,6 +344,35 @@ int dmxo_step_adam(dmxo* h, const void* const* grads, const int32_t* batch_sizes
   return dmxo_end(h, out_state);
 }
 
+// Window statistics over k consecutive state vectors (row-major k x n): per entry the mean and
+// the population standard deviation, by the two-pass definition in fp64; the flags entry (11)
+// gets the OR of the k flag words and spread 0. out has 2n entries: means, then deviations.
+// (Section "State representation": state vectors are built from metrics collected over k
+// iterations, as averages and standard deviations.)
+int dmxo_window_stats(const float* states, int k, int n, float* out) {
+  if (!states || !out || k < 1 || n <= iFlags) return kErrArg;
+  for (int i = 0; i < n; ++i) {
+    if (i == iFlags) {
+      unsigned f = 0;
+      for (int t = 0; t < k; ++t) f |= (unsigned)(int)states[(int64_t)t * n + i];
+      out[i] = (float)f;
+      out[n + i] = 0.0f;
+      continue;
+    }
+    double sum = 0.0;
+    for (int t = 0; t < k; ++t) sum += (double)states[(int64_t)t * n + i];
+    const double mean = sum / k;
+    double ss = 0.0;
+    for (int t = 0; t < k; ++t) {
+      const double d = (double)states[(int64_t)t * n + i] - mean;
+      ss += d * d;
+    }
+    out[i] = (float)mean;
+    out[n + i] = (float)std::sqrt(ss / k);
+  }
+  return kOk;
+}
+
 int dmxo_destroy(dmxo* h) {
   delete h;
   return kOk;

@@ -54,6 +54,8 @@ def lib():
         L.dmxo_begin_adam.argtypes = [vp, vp, f32, f32, f32, f32, i64]
         L.dmxo_range_adam.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp, i32]
         L.dmxo_step_adam.argtypes = [vp, vp, vp, vp, vp, vp, f32, f32, f32, f32, i64, vp, vp, i32]
+        L.dmxo_window_stats.argtypes = [vp, i32, i32, vp]
+        L.dmxo_window_stats.restype = i32
         for f in (L.dmxo_create, L.dmxo_state_len, L.dmxo_begin, L.dmxo_range, L.dmxo_end,
                   L.dmxo_step, L.dmxo_destroy, L.dmxo_begin_adam, L.dmxo_range_adam, L.dmxo_step_adam):
             f.restype = i32
@@ -69,6 +71,17 @@ class OracleError(RuntimeError):
 
 def _ptr(a: np.ndarray) -> int:
     return a.ctypes.data
+
+
+def window_stats(states: np.ndarray) -> np.ndarray:
+    """Mean and population std per entry over the rows of `states` (k x n float32); 2n floats."""
+    st = np.ascontiguousarray(states, dtype=np.float32)
+    k, n = st.shape
+    out = np.empty(2 * n, dtype=np.float32)
+    rc = lib().dmxo_window_stats(_ptr(st), k, n, _ptr(out))
+    if rc != 0:
+        raise OracleError(rc)
+    return out
 
 
 class Oracle:

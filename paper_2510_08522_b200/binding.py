@@ -20,7 +20,8 @@ ST_HDR = 16
 FLAG_NONFINITE, FLAG_G2_NONPOS, FLAG_COS_UNDEF, FLAG_SINGLE, FLAG_INTERNAL = 1, 2, 4, 8, 16
 
 EXPORTS = ("dmx_create", "dmx_state_len", "dmx_step", "dmx_step_adam", "dmx_step_host", "dmx_step_static", "dmx_set_profiling", "dmx_get_profile",
-           "dmx_launches_per_step", "dmx_destroy", "dmx_strerror", "dmx_last_cuda_error")
+           "dmx_launches_per_step", "dmx_destroy", "dmx_strerror", "dmx_last_cuda_error", "dmx_agg_create",
+           "dmx_agg_push", "dmx_agg_destroy")
 
 _lib = None
 
@@ -52,6 +53,12 @@ def lib():
         L.dmx_step_adam.restype = i32
         L.dmx_step_static.argtypes = [i32, i64, vp, i32, i32, vp, vp, vp, vp, f32, f32, vp, vp, vp]
         L.dmx_step_static.restype = i32
+        L.dmx_agg_create.argtypes = [i32, i32, ctypes.POINTER(vp)]
+        L.dmx_agg_create.restype = i32
+        L.dmx_agg_push.argtypes = [vp, vp, vp, ctypes.POINTER(i32), vp]
+        L.dmx_agg_push.restype = i32
+        L.dmx_agg_destroy.argtypes = [vp]
+        L.dmx_agg_destroy.restype = i32
         L.dmx_set_profiling.argtypes = [vp, i32]
         L.dmx_set_profiling.restype = i32
         L.dmx_get_profile.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(f32)]
@@ -128,6 +135,24 @@ def dmx_step_static(K, P, seg_offsets, grad_dtype, grad_ptrs, batch_sizes, param
     return lib().dmx_step_static(K, int(P), seg, len(seg_offsets) - 1, int(grad_dtype), gp, bs, int(params),
                                  int(momentum), float(lr), float(beta), int(prev_agg), int(out_state),
                                  int(stream) if stream else None)
+
+
+def dmx_agg_create(state_len, k):
+    """-> (code, handle) of a k-step window over state vectors of length state_len."""
+    a = ctypes.c_void_p()
+    rc = lib().dmx_agg_create(int(state_len), int(k), ctypes.byref(a))
+    return rc, a
+
+
+def dmx_agg_push(a, out_state, window_out, stream=0):
+    """-> (code, emitted). Raw device addresses; window_out has 2*state_len floats (mean, then std)."""
+    e = ctypes.c_int(0)
+    rc = lib().dmx_agg_push(a, int(out_state), int(window_out), ctypes.byref(e), int(stream) if stream else None)
+    return rc, e.value
+
+
+def dmx_agg_destroy(a) -> int:
+    return lib().dmx_agg_destroy(a)
 
 
 def dmx_set_profiling(h, on) -> int:
