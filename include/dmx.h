@@ -212,6 +212,57 @@ int dmx_agg_push(dmx_agg* a, const float* out_state, float* window_out, int* emi
 int dmx_agg_destroy(dmx_agg* a);
 
 /*
+ * dmx_ctl_decide — the controller's decision at the end of an adjustment cycle, on the device
+ * (Algorithm 1, the loops after the k training iterations: build each worker's state vector,
+ * evaluate the policy, apply the action within the batch-size limits, compute the reward).
+ * What the paper fixes: the action set {-100, -25, 0, +25, +100} and the update
+ * x_i <- max(min(x_i + a_i, x_max), x_min) (Section "Action space and batch size adjustment"),
+ * and the reward (Section "Reward function design")
+ *   r_i = Abar_i + alpha*max(0, dA_i) - beta_t*T_iter,i - delta*(log2 x_i - 5) - eta*(sigma2_norm + sigma_norm)
+ * with x_i the batch size used during the cycle; eta = 0 gives the SGD form. What it leaves open,
+ * and this library defines: the layout of the state vector and the policy network.
+ *
+ *   K, M, H        workers (1..DMX_MAX_WORKERS); caller-supplied metrics per worker
+ *                  (0..DMX_CTL_MAX_AUX: accuracy, accuracy gain, iteration time, network and system
+ *                  figures); hidden width of the policy network (1..DMX_CTL_MAX_HIDDEN)
+ *   state_len      length of the step's state vector (>= DMX_ST_HDR + K)
+ *   window         DEVICE, 2*state_len fp32: window means then deviations, as dmx_agg_push emits
+ *   aux            DEVICE, K x M fp32 row-major (may be NULL when M == 0)
+ *   batch          DEVICE, K int32: batch sizes used during the cycle (each >= 1)
+ *   weights        DEVICE, dmx_ctl_num_weights(M, H) fp32, row-major, in this order:
+ *                  W1 (H x F), c1 (H), W2 (H x H), c2 (H), W3 (5 x H), c3 (5), F = dmx_ctl_num_features(M)
+ *   col_acc, col_gain, col_titer   columns of aux holding Abar, dA, T_iter; -1 leaves the term out
+ *   alpha, beta_t, delta, eta      reward coefficients
+ *   b_min, b_max   batch-size limits (the paper uses 32 and 1024), 1 <= b_min <= b_max
+ *   uniforms       DEVICE, K fp32 in [0,1), or NULL. NULL: the action with the largest logit (lowest
+ *                  index on ties). Otherwise the action is drawn from softmax(logits): the smallest a
+ *                  whose cumulative probability exceeds uniforms[i] (the caller owns the generator)
+ *   next_batch     DEVICE out, K int32     action   DEVICE out, K int32 (index 0..4 into the action set)
+ *   reward         DEVICE out, K fp32      logits   DEVICE out, K x 5 fp32
+ *   features       DEVICE out, K x F fp32, or NULL
+ *
+ * State vector of worker i (F = M + 9 entries), with mean/dev the two halves of `window`:
+ *   aux[i][0..M), log2 x_i - 5, x_i*K / mean[B_TOTAL], mean[worker_sqnorm i] / mean[WMEAN_SQNORM],
+ *   mean[SIGMA_NORM], mean[SIGMA2_NORM], dev[SIGMA_NORM], mean[COS_PREV], dev[COS_PREV],
+ *   log2(1 + max(mean[GNS], 0) / mean[B_TOTAL])          (ratios with a zero denominator give 0)
+ * Policy: logits = W3 tanh(W2 tanh(W1 s + c1) + c2) + c3. Arithmetic is fp64, stored as fp32; the
+ * action is chosen from the fp32 logits as emitted.
+ * Asynchronous, one launch, no allocation, no host-device copy. Errors: DMX_ERR_ARG, DMX_ERR_CUDA.
+ */
+#define DMX_CTL_ACTIONS 5
+#define DMX_CTL_MAX_AUX 32
+#define DMX_CTL_MAX_HIDDEN 256
+#define DMX_CTL_LOCAL_EXTRA 3
+#define DMX_CTL_GLOBAL_FEATURES 6
+int dmx_ctl_num_features(int M);          /* M + 9, or DMX_ERR_ARG */
+int64_t dmx_ctl_num_weights(int M, int H);  /* H*F + H + H*H + H + 5*H + 5, or DMX_ERR_ARG */
+int dmx_ctl_decide(int K, int M, int H, int state_len, const float* window, const float* aux,
+                   const int32_t* batch, const float* weights, int col_acc, int col_gain, int col_titer,
+                   float alpha, float beta_t, float delta, float eta, int b_min, int b_max,
+                   const float* uniforms, int32_t* next_batch, int32_t* action, float* reward,
+                   float* logits, float* features, void* cuda_stream);
+
+/*
  * dmx_step_static — the same step without a handle and without any allocation.
  * (The paper has no counterpart: this entry point exists for the library's callers only.)
  *

@@ -21,7 +21,8 @@ FLAG_NONFINITE, FLAG_G2_NONPOS, FLAG_COS_UNDEF, FLAG_SINGLE, FLAG_INTERNAL = 1, 
 
 EXPORTS = ("dmx_create", "dmx_state_len", "dmx_step", "dmx_step_adam", "dmx_step_host", "dmx_step_static", "dmx_set_profiling", "dmx_get_profile",
            "dmx_launches_per_step", "dmx_destroy", "dmx_strerror", "dmx_last_cuda_error", "dmx_agg_create",
-           "dmx_agg_push", "dmx_agg_destroy")
+           "dmx_agg_push", "dmx_agg_destroy", "dmx_ctl_num_features", "dmx_ctl_num_weights", "dmx_ctl_decide")
+CTL_ACTIONS = (-100, -25, 0, 25, 100)
 
 _lib = None
 
@@ -59,6 +60,13 @@ def lib():
         L.dmx_agg_push.restype = i32
         L.dmx_agg_destroy.argtypes = [vp]
         L.dmx_agg_destroy.restype = i32
+        L.dmx_ctl_num_features.argtypes = [i32]
+        L.dmx_ctl_num_features.restype = i32
+        L.dmx_ctl_num_weights.argtypes = [i32, i32]
+        L.dmx_ctl_num_weights.restype = i64
+        L.dmx_ctl_decide.argtypes = [i32, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, f32, f32, f32, f32, i32, i32,
+                                     vp, vp, vp, vp, vp, vp, vp]
+        L.dmx_ctl_decide.restype = i32
         L.dmx_set_profiling.argtypes = [vp, i32]
         L.dmx_set_profiling.restype = i32
         L.dmx_get_profile.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(f32)]
@@ -153,6 +161,55 @@ def dmx_agg_push(a, out_state, window_out, stream=0):
 
 def dmx_agg_destroy(a) -> int:
     return lib().dmx_agg_destroy(a)
+
+
+def dmx_ctl_num_features(M) -> int:
+    return lib().dmx_ctl_num_features(int(M))
+
+
+def dmx_ctl_num_weights(M, H) -> int:
+    return lib().dmx_ctl_num_weights(int(M), int(H))
+
+
+def dmx_ctl_decide(K, M, H, state_len, window, aux, batch, weights, cols, coef, b_min, b_max, uniforms, next_batch,
+                   action, reward, logits, features, stream=0) -> int:
+    """The controller's decision for all K workers. Buffer arguments are raw device addresses (0 = NULL);
+    cols = (col_acc, col_gain, col_titer); coef = (alpha, beta_t, delta, eta)."""
+    def p(x):
+        return int(x) if x else None
+    return lib().dmx_ctl_decide(int(K), int(M), int(H), int(state_len), p(window), p(aux), p(batch), p(weights),
+                                int(cols[0]), int(cols[1]), int(cols[2]), float(coef[0]), float(coef[1]),
+                                float(coef[2]), float(coef[3]), int(b_min), int(b_max), p(uniforms), p(next_batch),
+                                p(action), p(reward), p(logits), p(features), p(stream))
+
+
+def ctl_decide(K, M, H, state_len, window, aux, batch, weights, cols=(-1, -1, -1), coef=(1.0, 0.0, 0.0, 0.0),
+               b_min=32, b_max=1024, uniforms=None, stream=None):
+    """Torch convenience over dmx_ctl_decide: device tensors in, a dict of new device tensors out
+    (next_batch, action: int32 [K]; reward: [K]; logits: [K, 5]; features: [K, F])."""
+    import torch
+    dev = window.device
+    F = dmx_ctl_num_features(M)
+    if F < 0 or weights.numel() != dmx_ctl_num_weights(M, H) or window.numel() != 2 * state_len or batch.numel() != K:
+        raise DmxError(ERR_ARG, "dmx_ctl_decide")
+    if (M > 0 and aux.numel() != K * M) or (uniforms is not None and uniforms.numel() != K):
+        raise DmxError(ERR_ARG, "dmx_ctl_decide")
+    for t, dt in ((window, torch.float32), (batch, torch.int32), (weights, torch.float32)):
+        if t.dtype != dt or not t.is_cuda or not t.is_contiguous():
+            raise DmxError(ERR_ARG, "dmx_ctl_decide (tensor)")
+    out = dict(next_batch=torch.empty(K, dtype=torch.int32, device=dev), action=torch.empty(K, dtype=torch.int32, device=dev),
+               reward=torch.empty(K, dtype=torch.float32, device=dev),
+               logits=torch.empty((K, len(CTL_ACTIONS)), dtype=torch.float32, device=dev),
+               features=torch.empty((K, F), dtype=torch.float32, device=dev))
+    if stream is None:
+        stream = torch.cuda.current_stream(dev).cuda_stream
+    rc = dmx_ctl_decide(K, M, H, state_len, window.data_ptr(), aux.data_ptr() if M > 0 else 0, batch.data_ptr(),
+                        weights.data_ptr(), cols, coef, b_min, b_max, uniforms.data_ptr() if uniforms is not None else 0,
+                        out["next_batch"].data_ptr(), out["action"].data_ptr(), out["reward"].data_ptr(),
+                        out["logits"].data_ptr(), out["features"].data_ptr(), stream)
+    if rc != OK:
+        raise DmxError(rc, "dmx_ctl_decide")
+    return out
 
 
 def dmx_set_profiling(h, on) -> int:
