@@ -247,7 +247,7 @@ def main():
     ap.add_argument("--workload", type=int, default=4, help="index into the workload table (default: the largest)")
     ap.add_argument("--also", type=int, default=3, help="second workload reported under 'also' (-1: none)")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-sample-elems", type=int, default=16 << 20, help="0: skip the CPU-baseline leg")
+    ap.add_argument("--cpu-sample-elems", type=int, default=128 << 20, help="0: skip the CPU-baseline leg")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "adam"],
                     help="update applied by the step (the metric's workload uses sgd)")
     ap.add_argument("--P", type=int, default=0, help="run the workload's structure at another size (profiling captures)")

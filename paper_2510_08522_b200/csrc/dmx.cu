@@ -59,7 +59,7 @@ struct dmx_handle {
   int nchunks = 0, nslots = 0, tile_group = 1;
   // device tables
   int64_t* seg_off = nullptr;
-  int32_t *tile_seg = nullptr, *cta_chunk0 = nullptr, *chunk_tile0 = nullptr, *chunk_ntiles = nullptr;
+  int32_t *tile_seg = nullptr, *chunk_stride = nullptr, *chunk_tile0 = nullptr, *chunk_ntiles = nullptr;
   int32_t *chunk_slot0 = nullptr, *seg_slots = nullptr, *unit_lo = nullptr, *unit_hi = nullptr, *seg_unit_ptr = nullptr;
   double2* segpart = nullptr;
   int nunits = 0;
@@ -67,7 +67,8 @@ struct dmx_handle {
   float* rows = nullptr;
   float2* slots = nullptr;
   double* colsum = nullptr;
-  unsigned* flags = nullptr;  // [0] ticket, [1] err
+  unsigned* flags = nullptr;  // [0] ticket, [1] err, [2] and [3] chunk counters of even and odd steps
+  unsigned step_parity = 0;   // which chunk counter the next step draws from
   // optional per-kernel timing
   bool profiling = false, profiled = false;
   cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
@@ -101,12 +102,32 @@ Plan pick_direct(int K) {
 // Pipelined (bulk-copy ring) kernels. Ring geometry: 7 consumer warps + the producer warp = 8
 // warps, so that a thread may use up to 255 registers (9 warps are allocated as 12 and cap it
 // at 168, which spilled at K = 32); 4 gradient streams per 14 KB stage (smaller stages lose to
-// the per-stage synchronisation, larger ones leave too few in flight); as many stages as fit
-// beside one state stage (a second state stage measured 2-3 % slower on B200).
+// the per-stage synchronisation, larger ones leave too few in flight).
+// The producer runs at most NSS tiles ahead of the consumers (a tile's state stage is freed when
+// the consumers have read it), so the bytes in flight per SM are min(ring, NSS tiles). With many
+// workers one tile already fills the ring and one state stage is best (a second one measured 2-3 %
+// slower at K = 32); with few workers a tile is small, and one state stage left only ~40 KB per
+// SM in flight (0.76 of the copy rate at K = 8): there the ring is split into as many whole tiles
+// (gradient stages + a state stage each) as fit.
+template <int KT, bool BF16, bool ADAM>
+struct Ring {
+  static constexpr int CW = 7, G = 4;
+  static constexpr int kStage = CW * 32 * 16 * G;                                   // bytes of a gradient stage
+  static constexpr int kState = CW * 32 * (BF16 ? 8 : 4) * 4 * (ADAM ? 4 : 3);      // bytes of a state stage
+  static constexpr int kTile = (KT + G - 1) / G * kStage + kState;                  // shared memory of one tile
+  static constexpr int kAhead = 240 * 1024 / kTile;
+  static constexpr int NSS = kAhead < 1 ? 1 : (kAhead > 8 ? 8 : kAhead);
+  static constexpr int kRed = (int)((sizeof(dmx::RedArea<KT, CW>) + 15) / 16 * 16);
+  static constexpr int kFit = (227 * 1024 - NSS * (kState + 16) - kRed - 128) / (kStage + 16);
+  static constexpr int kTuned = BF16 ? (ADAM ? 12 : 13) : 14;                       // measured best with one state stage
+  static constexpr int NSTAGE = NSS == 1 ? kTuned : (kFit > 32 ? 32 : kFit);
+  typedef dmx::PipeCfg<KT, BF16, CW, G, NSTAGE, NSS, ADAM> Cfg;
+};
+
 template <int KT, bool BF16>
 Plan pipe_plan() {
-  typedef dmx::PipeCfg<KT, BF16, 7, 4, BF16 ? 13 : 14, 1, false> C;
-  typedef dmx::PipeCfg<KT, BF16, 7, 4, BF16 ? 12 : 14, 1, true> CA;
+  typedef typename Ring<KT, BF16, false>::Cfg C;
+  typedef typename Ring<KT, BF16, true>::Cfg CA;
   static_assert(C::T == CA::T && C::THREADS == CA::THREADS, "both updates share the tile tables");
   Plan p;
   p.kernel = dmx::pipe_kernel<C>;
@@ -129,7 +150,7 @@ Plan pick_pipe(int K) {
 
 void free_handle(dmx_handle* h) {
   if (!h) return;
-  cudaFree(h->seg_off); cudaFree(h->tile_seg); cudaFree(h->cta_chunk0); cudaFree(h->chunk_tile0);
+  cudaFree(h->seg_off); cudaFree(h->tile_seg); cudaFree(h->chunk_stride); cudaFree(h->chunk_tile0);
   cudaFree(h->chunk_ntiles); cudaFree(h->chunk_slot0); cudaFree(h->seg_slots); cudaFree(h->unit_lo);
   cudaFree(h->unit_hi); cudaFree(h->seg_unit_ptr); cudaFree(h->segpart);
   cudaFree(h->rows); cudaFree(h->slots); cudaFree(h->colsum); cudaFree(h->flags);
@@ -189,17 +210,24 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   const int want = env_int("DMX_CTAS_PER_SM", 0);   // tuning knob: resident CTAs per SM (0 = all that fit)
   if (want > 0 && want < occ) occ = want;
   const int64_t ntiles = (P + plan.tile - 1) / plan.tile;
-  // Tiles are dealt round robin in groups of R consecutive tiles: group g belongs to CTA
-  // g mod grid. A CTA's tiles are cut into chunks of about `DMX_CHUNK_TILES` tiles so that fp32
-  // per-thread partials stay short. The cut is a function of (P, tile, grid, R) only, so
-  // results are reproducible on a given device.
-  // Groups of 4 tiles measured 0.5-1 % faster than single tiles on the large workloads, but a
-  // CTA's share is a whole number of groups: keep at least 64 groups per CTA so that the
-  // imbalance stays below ~1.5 % (small problems fall back to groups of 2 or 1).
+  // Tiles are taken in groups of R consecutive tiles; a chunk is a few groups, interleaved with
+  // the other chunks of its wave: chunk l of a wave of n chunks that starts at group g0 holds
+  // groups g0+l, g0+l+n, ... A full wave has one chunk per CTA. Chunks are about a sixth of a
+  // CTA's share, at most `DMX_CHUNK_TILES` tiles (so that fp32 per-thread partials stay short) and
+  // at least 8: SM speeds drift during a kernel, and on the mid-sized workloads 16-tile chunks
+  // measured 3-4 % faster than 32-tile ones, while below 8 tiles the per-chunk work shows. Once
+  // fewer than two such waves remain, every wave takes about half of what is left, down to a
+  // minimum chunk, and the last wave splits its rest evenly, so that the CTAs finish together
+  // under the dynamic schedule. The list is a function of (P, tile, grid, R) only and a chunk's
+  // sums do not depend on the CTA that computes it: results are reproducible on a given device.
+  // Groups of 4 tiles measured 0.5-1 % faster than single tiles on the large workloads, groups
+  // of 2 about 1 % faster on the mid-sized ones.
   const int64_t sm_ctas = (int64_t)prop.multiProcessorCount * occ;
-  const int auto_R = ntiles >= 4 * 64 * sm_ctas ? 4 : (ntiles >= 2 * 64 * sm_ctas ? 2 : 1);
+  const int auto_R = ntiles >= 4 * 64 * sm_ctas ? 4 : (ntiles >= 32 * sm_ctas ? 2 : 1);
   const int R = std::max(1, std::min(env_int("DMX_TILE_GROUP", auto_R), 1 << 16));   // tuning knob: tiles per group
-  const int chunk_groups = std::max(1, env_int("DMX_CHUNK_TILES", 32) / R);
+  const int64_t share = (ntiles + sm_ctas - 1) / sm_ctas;                            // tiles per CTA
+  const int auto_chunk = (int)std::max<int64_t>(8, std::min<int64_t>(32, share / 6));
+  const int chunk_groups = std::max(1, env_int("DMX_CHUNK_TILES", auto_chunk) / R);
   const int64_t ngroups = (ntiles + R - 1) / R;
   plan.grid = (int)std::min<int64_t>((int64_t)prop.multiProcessorCount * occ, ngroups);
   h->plan = plan;
@@ -215,18 +243,35 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
       tile_seg[(size_t)t] = s | (seg_offsets[s + 1] < j1 && s < S - 1 ? dmx::kTileBoundaryBit : 0);
     }
   }
-  std::vector<int32_t> cta_chunk0(grid + 1), chunk_tile0, chunk_ntiles, chunk_slot0;
-  for (int b = 0; b < grid; ++b) {
-    cta_chunk0[b] = (int32_t)chunk_tile0.size();
-    const int64_t nb = (ngroups - b + grid - 1) / grid;    // groups b, b+grid, ...
-    for (int64_t i = 0; i < nb; i += chunk_groups) {
-      const int64_t g0 = b + i * grid, ng = std::min<int64_t>(chunk_groups, nb - i);
-      const int64_t glast = g0 + (ng - 1) * grid;            // the last group may be cut short by ntiles
-      chunk_tile0.push_back((int32_t)(g0 * R));
-      chunk_ntiles.push_back((int32_t)((ng - 1) * R + std::min<int64_t>(R, ntiles - glast * R)));
+  std::vector<int32_t> chunk_tile0, chunk_ntiles, chunk_stride, chunk_slot0;
+  // smallest chunk: about 192 KB of streamed bytes (a few microseconds of one SM), so that the
+  // per-chunk work (the draw, the reduction flush) stays small beside it
+  const int64_t group_bytes = (int64_t)R * plan.tile * ((int64_t)K * (grad_dtype == DMX_BF16 ? 2 : 4) + 24);
+  const int64_t min_groups = std::min<int64_t>(chunk_groups, std::max<int64_t>(1, (192 * 1024 + group_bytes - 1) / group_bytes));
+  for (int64_t g0 = 0; g0 < ngroups;) {
+    const int64_t rem = ngroups - g0;
+    const int64_t ng = rem <= 2 * min_groups * (int64_t)grid
+                           ? (rem + grid - 1) / grid      // the last wave: what is left, split evenly
+                           : std::max<int64_t>(min_groups, std::min<int64_t>(chunk_groups, rem / (2 * (int64_t)grid)));
+    const int64_t nl = std::min<int64_t>(grid, (rem + ng - 1) / ng);
+    const int64_t wave = std::min<int64_t>(rem, nl * ng);      // groups g0 .. g0+wave-1, lane l takes g0+l, g0+l+nl, ...
+    for (int64_t l = 0; l < nl; ++l) {
+      const int64_t n_l = (wave - l + nl - 1) / nl;
+      const int64_t glast = g0 + l + (n_l - 1) * nl;            // only the very last group may be cut short by ntiles
+      chunk_tile0.push_back((int32_t)((g0 + l) * R));
+      chunk_ntiles.push_back((int32_t)((n_l - 1) * R + std::min<int64_t>(R, ntiles - glast * R)));
+      chunk_stride.push_back((int32_t)(nl * R));
     }
+    g0 += wave;
   }
-  cta_chunk0[grid] = (int32_t)chunk_tile0.size();
+  // The chunk that ends the list holds the last tile. If that tile is ragged it goes through the
+  // guarded plain-load path, several times slower than a full tile: drawn last it would extend
+  // the kernel by that much (8 % at P = 25.6 M), so it is drawn first instead.
+  if (P % plan.tile != 0 && chunk_tile0.size() > 1) {
+    std::rotate(chunk_tile0.begin(), chunk_tile0.end() - 1, chunk_tile0.end());
+    std::rotate(chunk_ntiles.begin(), chunk_ntiles.end() - 1, chunk_ntiles.end());
+    std::rotate(chunk_stride.begin(), chunk_stride.end() - 1, chunk_stride.end());
+  }
   const int nchunks = (int)chunk_tile0.size();
   // Enumerate, with the kernel's own rules, the (V, N) entries every chunk emits: a new entry
   // whenever the running segment changes between tiles, at every boundary crossed inside a
@@ -237,7 +282,7 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
     chunk_slot0[c] = (int32_t)slot_seg.size();
     int cur = -1;
     for (int i = 0; i < chunk_ntiles[c]; ++i) {
-      const int64_t t = chunk_tile0[c] + (int64_t)(i / R) * R * grid + i % R;
+      const int64_t t = chunk_tile0[c] + (int64_t)(i / R) * chunk_stride[c] + i % R;
       const int64_t j1 = std::min<int64_t>((t + 1) * plan.tile, P);
       const int s0 = tile_seg[(size_t)t] & (dmx::kTileBoundaryBit - 1);
       if (s0 != cur) {
@@ -272,7 +317,7 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   h->nchunks = nchunks; h->nslots = (int)nslots; h->nunits = (int)unit_lo.size();
 
   std::vector<int64_t> seg(seg_offsets, seg_offsets + S + 1);
-  bool ok = upload(seg, &h->seg_off) && upload(tile_seg, &h->tile_seg) && upload(cta_chunk0, &h->cta_chunk0) &&
+  bool ok = upload(seg, &h->seg_off) && upload(tile_seg, &h->tile_seg) && upload(chunk_stride, &h->chunk_stride) &&
             upload(chunk_tile0, &h->chunk_tile0) && upload(chunk_ntiles, &h->chunk_ntiles) &&
             upload(chunk_slot0, &h->chunk_slot0) && upload(seg_slots, &h->seg_slots) && upload(unit_lo, &h->unit_lo) &&
             upload(unit_hi, &h->unit_hi) && upload(seg_unit_ptr, &h->seg_unit_ptr);
@@ -280,8 +325,8 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   ok = ok && cuda_ok(cudaMalloc((void**)&h->rows, (size_t)nchunks * (K + 4) * sizeof(float)));
   ok = ok && cuda_ok(cudaMalloc((void**)&h->slots, (size_t)std::max<int64_t>(nslots, 1) * sizeof(float2)));
   ok = ok && cuda_ok(cudaMalloc((void**)&h->colsum, (size_t)(K + 4) * sizeof(double)));
-  ok = ok && cuda_ok(cudaMalloc((void**)&h->flags, 2 * sizeof(unsigned)));
-  ok = ok && cuda_ok(cudaMemset(h->flags, 0, 2 * sizeof(unsigned)));
+  ok = ok && cuda_ok(cudaMalloc((void**)&h->flags, 4 * sizeof(unsigned)));
+  ok = ok && cuda_ok(cudaMemset(h->flags, 0, 4 * sizeof(unsigned)));
   ok = ok && cuda_ok(cudaDeviceSynchronize());
   if (!ok) {
     const bool nomem = g_last_cuda == (int)cudaErrorMemoryAllocation;
@@ -366,8 +411,10 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
     A.c2 = (float)(1.0 / (1.0 - std::pow((double)ap->beta2, (double)ap->t)));
   }
   A.K = K; A.S = h->S; A.P = h->P;
-  A.tile_group = h->tile_group; A.group_stride = h->tile_group * h->plan.grid; A.nchunks = h->nchunks;
-  A.seg_off = h->seg_off; A.tile_seg = h->tile_seg; A.cta_chunk0 = h->cta_chunk0; A.chunk_tile0 = h->chunk_tile0;
+  A.tile_group = h->tile_group; A.nchunks = h->nchunks;
+  // the step's chunk counter is zero: the previous step's kernel reset it while it drew from the other one
+  A.next_chunk = h->flags + 2 + h->step_parity; A.next_chunk_reset = h->flags + 2 + (h->step_parity ^ 1u);
+  A.seg_off = h->seg_off; A.tile_seg = h->tile_seg; A.chunk_stride = h->chunk_stride; A.chunk_tile0 = h->chunk_tile0;
   A.chunk_ntiles = h->chunk_ntiles; A.chunk_slot0 = h->chunk_slot0;
   A.rows = h->rows; A.slots = h->slots; A.err = h->flags + 1;
 
@@ -383,6 +430,7 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
   if (ap) h->plan.kernel_adam<<<h->plan.grid, h->plan.threads, h->plan.smem_adam, stream>>>(A);
   else h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A);
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
+  h->step_parity ^= 1u;   // only a step that was enqueued consumes its counter
   if (prof && !cuda_ok(cudaEventRecord(h->ev[1], stream))) return DMX_ERR_CUDA;
   const int funits = K + 2 + 2 * F.adam + h->nunits;   // one warp per chunk-row column and per segment unit
   const int fblocks = (funits + dmx::kFinalWarps - 1) / dmx::kFinalWarps;

@@ -13,15 +13,21 @@
 // cancellation is between noise-sized terms only. The arithmetic runs on pairs of fp32
 // values with the packed f32x2 instructions of sm_100 (each lane IEEE fp32, round to nearest).
 //
-// Work layout. The parameter range is cut into tiles of T elements, dealt to the CTAs round
-// robin in groups of R consecutive tiles (group g belongs to CTA g mod grid), so at any moment
-// the CTAs sweep a compact window of every stream (DRAM sees a few dozen linear sweeps instead
-// of thousands of scattered 4 KB reads). A CTA's tiles are grouped into chunks of a few dozen.
+// Work layout. The parameter range is cut into tiles of T elements, taken in groups of R
+// consecutive tiles. The unit of work is a chunk: a few groups, interleaved with the other
+// chunks of its wave (chunk l of a wave of n chunks holds groups first+l, first+l+n, ...), so
+// that the CTAs working on one wave sweep a compact window of every stream (DRAM sees a few
+// dozen linear sweeps instead of thousands of scattered 4 KB reads). The chunk list is fixed by
+// the host; waves shrink towards the end of the range. The pipelined kernel hands chunks to its
+// CTAs dynamically (an atomic counter): SMs do not all stream at the same rate, and a static
+// split left the fast ones idle for 3-12 % of the kernel.
 //
 // Reductions are deterministic: per-thread fp32 partials over a chunk, warp shuffles, a
 // fixed-order sum over the warps, one scratch row per chunk and one scratch slot per
 // (chunk, run of tiles in one segment), then an fp64 fixed-order second level in the
-// finalize kernel. There are no floating-point atomics and no waits between CTAs.
+// finalize kernel. A chunk's sums do not depend on which CTA computes it, so results are
+// bitwise reproducible under the dynamic schedule. There are no floating-point atomics and no
+// waits between CTAs.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -46,15 +52,16 @@ struct StepArgs {
   float beta2, eps, omb1, omb2, c1, c2;   // Adam: beta2, eps, 1-beta1, 1-beta2, 1/(1-beta1^t), 1/(1-beta2^t)
   int K, S;
   int64_t P;
-  int tile_group;              // R: tiles are dealt to the CTAs in groups of R consecutive tiles
-  int group_stride;            // = R * grid: distance between a CTA's successive groups
+  int tile_group;              // R: consecutive tiles per group
   int nchunks;
+  unsigned* next_chunk;        // dynamic schedule: the counter of this step (zero at launch)
+  unsigned* next_chunk_reset;  // the counter of the following step: CTA 0 zeroes it
   const int64_t* seg_off;      // S+1
   const int32_t* tile_seg;     // ntiles: segment of the tile's first element; kTileBoundaryBit set
                                //         when a segment boundary lies strictly inside the tile
-  const int32_t* cta_chunk0;   // grid+1: chunks [cta_chunk0[b], cta_chunk0[b+1]) belong to CTA b
   const int32_t* chunk_tile0;  // nchunks: first tile of the chunk
-  const int32_t* chunk_ntiles; // nchunks: tiles in the chunk (tile0, tile0+stride, ...)
+  const int32_t* chunk_ntiles; // nchunks: tiles in the chunk
+  const int32_t* chunk_stride; // nchunks: tiles between the starts of the chunk's successive groups
   const int32_t* chunk_slot0;  // nchunks: first (V,N) slot of the chunk
   float* rows;                 // (K+4) x nchunks, one column after the other: q_k..., c, pp, and (Adam) su, su2
   float2* slots;               // nslots: (V partial, N partial), in the order the chunk emits them
@@ -102,10 +109,10 @@ __device__ __forceinline__ u64 mul2(u64 a, u64 b) {
   u64 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d;
 }
 
-// i-th tile of a chunk whose first tile is t0
-__device__ __forceinline__ int tile_of(const StepArgs& A, int t0, int i) {
+// i-th tile of a chunk whose first tile is t0 and whose groups start `stride` tiles apart
+__device__ __forceinline__ int tile_of(const StepArgs& A, int t0, int stride, int i) {
   const int g = i / A.tile_group;
-  return t0 + g * A.group_stride + (i - g * A.tile_group);
+  return t0 + g * stride + (i - g * A.tile_group);
 }
 
 __device__ __forceinline__ float sqrt_approx(float x) { float r; asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
@@ -182,62 +189,81 @@ __device__ __forceinline__ void named_sync(int bar_id) {
   asm volatile("bar.sync %0, %1;" :: "r"(bar_id), "r"(NW * 32) : "memory");
 }
 
+// Barrier among the NW warps that take part in the reductions (hardware named barrier 1).
+template <int NW>
+struct BarSync {
+  __device__ __forceinline__ void sync() { named_sync<NW>(1); }
+};
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
 }
 
-// Shared-memory work area of the reductions (used by the NW participating warps only).
+// Shared-memory work area of the reductions (used by the NW participating warps only). Two
+// copies, used by alternate chunks: a chunk ends with ONE barrier (after the warps have written
+// their partials), and the warps that leave it first may fill the other copy for the next chunk
+// while the slower ones still read this one. A copy is reused two chunks later, i.e. after the
+// next chunk's barrier, which every thread reaches only after it has finished reading.
 template <int KT, int NW>
 struct RedArea {
-  float rows[NW][KT + 4];
-  float2 seg[kSegBuf][NW];
+  float rows[2][NW][KT + 4];
+  float2 seg[2][kSegBuf][NW];
 };
 
-// Per-chunk segment bookkeeping; identical in every participating thread.
+// Segment bookkeeping; identical in every participating thread.
 struct SegState {
   int cur;      // segment the running (vs, ns) belong to; -1 before the chunk's first tile
   int nent;     // entries emitted so far in this chunk
   int nbuf;     // of which still buffered in shared memory
+  int par;      // which copy of the work area the current chunk uses
+  __device__ __forceinline__ void begin_chunk() { cur = -1; nent = 0; nbuf = 0; }
 };
 
-// Write the buffered segment partials to their slots (fixed order over the warps).
+// Sum the buffered segment partials over the warps (fixed order) into their slots.
 template <int KT, int NW>
-__device__ __forceinline__ void seg_drain(RedArea<KT, NW>* R, SegState& st, float2* chunk_slots, int bar_id) {
-  named_sync<NW>(bar_id);
+__device__ __forceinline__ void seg_write(RedArea<KT, NW>* R, const SegState& st, float2* chunk_slots) {
   for (int e = threadIdx.x; e < st.nbuf; e += NW * 32) {
     float v = 0.f, n = 0.f;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) { const float2 t = R->seg[e][w]; v += t.x; n += t.y; }
+    for (int w = 0; w < NW; ++w) { const float2 t = R->seg[st.par][e][w]; v += t.x; n += t.y; }
     chunk_slots[st.nent - st.nbuf + e] = make_float2(v, n);
   }
-  named_sync<NW>(bar_id);
+}
+
+// The buffer is full in the middle of a chunk (more than kSegBuf segment boundaries in it):
+// empty it between two barriers.
+template <int KT, int NW, class SY>
+__device__ __forceinline__ void seg_drain(RedArea<KT, NW>* R, SegState& st, float2* chunk_slots, SY& sy) {
+  sy.sync();
+  seg_write<KT, NW>(R, st, chunk_slots);
+  sy.sync();
   st.nbuf = 0;
 }
 
 // Close the running (vs, ns) as the next entry of the chunk: a warp reduction and one
 // shared-memory store per warp; no block barrier unless the shared buffer is full.
-template <int KT, int VEC, int NW>
+template <int KT, int VEC, int NW, class SY>
 __device__ __forceinline__ void seg_entry(Acc<KT, VEC>& a, RedArea<KT, NW>* R, SegState& st, float2* chunk_slots,
-                                          int bar_id, int wid, int lane) {
+                                          SY& sy, int wid, int lane) {
   const float v = warp_sum(a.vs), n = warp_sum(a.ns);
-  if (lane == 0) R->seg[st.nbuf][wid] = make_float2(v, n);
+  if (lane == 0) R->seg[st.par][st.nbuf][wid] = make_float2(v, n);
   a.vs = 0.f; a.ns = 0.f;
   ++st.nbuf; ++st.nent;
-  if (st.nbuf == kSegBuf) seg_drain<KT, NW>(R, st, chunk_slots, bar_id);
+  if (st.nbuf == kSegBuf) seg_drain<KT, NW>(R, st, chunk_slots, sy);
 }
 
 // Attribute the tile's per-element (d, g^2) to segments. `tseg` is the tile's table entry.
 // The host enumerates the entries of a chunk with the same rules (see build_tables).
-template <int KT, int VEC, int NW>
+template <int KT, int VEC, int NW, class SY>
 __device__ __forceinline__ void segment_accumulate(Acc<KT, VEC>& a, const StepArgs& A, const float* dv,
                                                    const float* nv, int64_t jt, int64_t tile_begin,
                                                    int64_t tile_end, int tseg, RedArea<KT, NW>* R, SegState& st,
-                                                   float2* chunk_slots, int bar_id, int wid, int lane) {
+                                                   float2* chunk_slots, SY& sy, int wid, int lane) {
   const int s0 = tseg & (kTileBoundaryBit - 1);
   if (s0 != st.cur) {
-    if (st.cur >= 0) seg_entry<KT, VEC, NW>(a, R, st, chunk_slots, bar_id, wid, lane);
+    if (st.cur >= 0) seg_entry<KT, VEC, NW>(a, R, st, chunk_slots, sy, wid, lane);
     st.cur = s0;
   }
   if (!(tseg & kTileBoundaryBit)) {
@@ -253,7 +279,7 @@ __device__ __forceinline__ void segment_accumulate(Acc<KT, VEC>& a, const StepAr
       const int64_t j = jt + e;
       if (j >= lo && j < next_bound) { a.vs += dv[e]; a.ns += nv[e]; }
     }
-    seg_entry<KT, VEC, NW>(a, R, st, chunk_slots, bar_id, wid, lane);
+    seg_entry<KT, VEC, NW>(a, R, st, chunk_slots, sy, wid, lane);
     lo = next_bound;
     ++st.cur;
     next_bound = A.seg_off[st.cur + 1];
@@ -264,11 +290,12 @@ __device__ __forceinline__ void segment_accumulate(Acc<KT, VEC>& a, const StepAr
   }
 }
 
-// End of a chunk: last segment entry, drain, then q_k, c, pp -> the chunk's scratch row.
-template <int KT, int VEC, int NW, bool ADAM = false>
+// End of a chunk: last segment entry, then the segment partials -> their slots and q_k, c, pp ->
+// the chunk's scratch row.
+template <int KT, int VEC, int NW, bool ADAM, class SY>
 __device__ __forceinline__ void flush_chunk(Acc<KT, VEC>& a, const StepArgs& A, RedArea<KT, NW>* R, SegState& st,
-                                            int chunk, float2* chunk_slots, int bar_id, int wid, int lane) {
-  if (st.cur >= 0) seg_entry<KT, VEC, NW>(a, R, st, chunk_slots, bar_id, wid, lane);
+                                            int chunk, float2* chunk_slots, SY& sy, int wid, int lane) {
+  if (st.cur >= 0) seg_entry<KT, VEC, NW>(a, R, st, chunk_slots, sy, wid, lane);
   constexpr int NV = KT + 2 + (ADAM ? 2 : 0);
   float v[NV];
 #pragma unroll
@@ -277,18 +304,19 @@ __device__ __forceinline__ void flush_chunk(Acc<KT, VEC>& a, const StepArgs& A, 
   if constexpr (ADAM) { v[KT + 2] = warp_sum(a.su); v[KT + 3] = warp_sum(a.su2); }
   if (lane == 0) {
 #pragma unroll
-    for (int i = 0; i < NV; ++i) R->rows[wid][i] = v[i];
+    for (int i = 0; i < NV; ++i) R->rows[st.par][wid][i] = v[i];
   }
-  seg_drain<KT, NW>(R, st, chunk_slots, bar_id);   // its first barrier also publishes rows[][]
+  sy.sync();                                       // the chunk's only barrier: every warp's partials are in place
+  seg_write<KT, NW>(R, st, chunk_slots);
   const int t = wid * 32 + lane;
   if (t < NV) {
     float s = 0.f;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) s += R->rows[w][t];
+    for (int w = 0; w < NW; ++w) s += R->rows[st.par][w][t];
     if (t < KT) { if (t < A.K) A.rows[(int64_t)t * A.nchunks + chunk] = s; }
     else A.rows[(int64_t)(A.K + t - KT) * A.nchunks + chunk] = s;
   }
-  named_sync<NW>(bar_id);                          // rows[][] may be rewritten by the next chunk
+  st.par ^= 1;                                     // the next chunk fills the other copy
   a.reset_chunk();
 }
 
@@ -436,13 +464,15 @@ direct_kernel(const __grid_constant__ StepArgs A) {
   const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
   Acc<KT, VEC> a;
   a.reset_chunk();
-  const int c_begin = A.cta_chunk0[blockIdx.x], c_end = A.cta_chunk0[blockIdx.x + 1];
-  for (int c = c_begin; c < c_end; ++c) {
-    const int t0 = A.chunk_tile0[c], nt = A.chunk_ntiles[c];
+  BarSync<NW> sy;
+  SegState st; st.par = 0;
+  // chunks are dealt statically here: chunk c belongs to CTA c mod grid
+  for (int c = blockIdx.x; c < A.nchunks; c += gridDim.x) {
+    const int t0 = A.chunk_tile0[c], nt = A.chunk_ntiles[c], cstride = A.chunk_stride[c];
     float2* chunk_slots = A.slots + A.chunk_slot0[c];
-    SegState st; st.cur = -1; st.nent = 0; st.nbuf = 0;
+    st.begin_chunk();
     for (int i = 0; i < nt; ++i) {
-      const int t = tile_of(A, t0, i);
+      const int t = tile_of(A, t0, cstride, i);
       const int tseg = A.tile_seg[t];
       const int64_t tile_begin = (int64_t)t * T;
       const int64_t jt = tile_begin + (int64_t)threadIdx.x * VEC;
@@ -454,9 +484,9 @@ direct_kernel(const __grid_constant__ StepArgs A) {
         tile_end = A.P;
         direct_tile<KT, BF16, true, U, ADAM>(a, A, jt, dv, nv);
       }
-      segment_accumulate<KT, VEC, NW>(a, A, dv, nv, jt, tile_begin, tile_end, tseg, &R, st, chunk_slots, 1, wid, lane);
+      segment_accumulate<KT, VEC, NW>(a, A, dv, nv, jt, tile_begin, tile_end, tseg, &R, st, chunk_slots, sy, wid, lane);
     }
-    flush_chunk<KT, VEC, NW, ADAM>(a, A, &R, st, c, chunk_slots, 1, wid, lane);
+    flush_chunk<KT, VEC, NW, ADAM>(a, A, &R, st, c, chunk_slots, sy, wid, lane);
   }
 }
 
@@ -634,6 +664,22 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   return r;
 }
 
+// Barrier among the consumer warps built on an mbarrier (one arrival per warp), so that its
+// wait is bounded like every other wait of this kernel: if a warp has left after a failed wait,
+// the others time out, raise the error word and go on instead of hanging in a hardware barrier.
+struct MbarSync {
+  uint32_t bar, phase;
+  volatile uint32_t* give_up;
+  unsigned* err;
+  int lane;
+  __device__ __forceinline__ void sync() {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+    (void)mbar_wait(bar, phase, give_up, err);
+    phase ^= 1u;
+  }
+};
+
 template <int KT_, bool BF16_, int CW_, int G_, int NSTAGE_, int NSS_, bool ADAM_ = false>
 struct PipeCfg {
   static constexpr int KT = KT_, CW = CW_, G = G_, NSTAGE = NSTAGE_, NSS = NSS_;
@@ -650,8 +696,10 @@ struct PipeCfg {
   static constexpr int RING = NSTAGE * STAGE;
   static constexpr int SRING = NSS * SSTAGE;
   static constexpr int RED = (int)((sizeof(RedArea<KT, CW>) + 15) / 16 * 16);
-  static constexpr int NBAR = 2 * NSTAGE + 2 * NSS;
-  static constexpr size_t SMEM = (size_t)RING + SRING + RED + NBAR * 8 + 16;
+  static constexpr int QN = 4;                       // chunk descriptors in flight from the producer to the consumers
+  static constexpr int NBAR = 2 * NSTAGE + 2 * NSS + 2 * QN + 1;
+  static constexpr int TAIL = 16 + QN * 32;          // give-up word, chunk queue (8 ints per entry)
+  static constexpr size_t SMEM = (size_t)RING + SRING + RED + NBAR * 8 + TAIL;
   static_assert(G >= 1 && G <= 32, "one producer lane per stream of a stage");
   static_assert(NSTAGE <= 32 && NSS <= 32, "stage masks are 32 bits wide");
   static_assert(SMEM <= 227 * 1024, "ring does not fit in shared memory");
@@ -659,27 +707,32 @@ struct PipeCfg {
 
 template <class C>
 __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_constant__ StepArgs A) {
-  constexpr int KT = C::KT, VEC = C::VEC, CW = C::CW, G = C::G, NSTAGE = C::NSTAGE, NSS = C::NSS, T = C::T;
+  constexpr int KT = C::KT, VEC = C::VEC, CW = C::CW, G = C::G, NSTAGE = C::NSTAGE, NSS = C::NSS, T = C::T, QN = C::QN;
   constexpr bool BF16 = C::BF16, ADAM = C::ADAM;
   extern __shared__ __align__(128) unsigned char smem[];
   const uint32_t ring = smem_u32(smem);
   const uint32_t sring = ring + C::RING;
   RedArea<KT, CW>* R = reinterpret_cast<RedArea<KT, CW>*>(smem + C::RING + C::SRING);
   const uint32_t bars = sring + C::SRING + C::RED;
-  volatile uint32_t* give_up = reinterpret_cast<volatile uint32_t*>(smem + C::RING + C::SRING + C::RED + C::NBAR * 8);
-  // barrier i: full_g[i] = bars + 8 i ; empty_g[i] = bars + 8 (NSTAGE + i)
-  //            full_s[i] = bars + 8 (2 NSTAGE + i) ; empty_s[i] = bars + 8 (2 NSTAGE + NSS + i)
+  unsigned char* tail = smem + C::RING + C::SRING + C::RED + C::NBAR * 8;
+  volatile uint32_t* give_up = reinterpret_cast<volatile uint32_t*>(tail);
+  volatile int* queue = reinterpret_cast<volatile int*>(tail + 16);   // entry: chunk (-1: none left), first tile,
+                                                                       // tiles, group stride, first slot
+  // barriers, 8 bytes each: full_g[NSTAGE], empty_g[NSTAGE], full_s[NSS], empty_s[NSS],
+  // full_q[QN], empty_q[QN], and the consumers' own barrier
   const uint32_t full_g = bars, empty_g = bars + 8 * NSTAGE, full_s = bars + 16 * NSTAGE, empty_s = full_s + 8 * NSS;
+  const uint32_t full_q = empty_s + 8 * NSS, empty_q = full_q + 8 * QN, csync = empty_q + 8 * QN;
   const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int i = 0; i < NSTAGE; ++i) { mbar_init(full_g + 8 * i, 1); mbar_init(empty_g + 8 * i, CW); }
     for (int i = 0; i < NSS; ++i) { mbar_init(full_s + 8 * i, 1); mbar_init(empty_s + 8 * i, CW); }
+    for (int i = 0; i < QN; ++i) { mbar_init(full_q + 8 * i, 1); mbar_init(empty_q + 8 * i, CW); }
+    mbar_init(csync, CW);
     *give_up = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
-  const int c_begin = A.cta_chunk0[blockIdx.x], c_end = A.cta_chunk0[blockIdx.x + 1];
   constexpr int ESZ = BF16 ? 2 : 4;
 
   if (wid == CW) {
@@ -687,15 +740,51 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
     // The whole warp takes part: every lane waits for the stage to be free, lane 0 arms the
     // barrier with the byte count, then lane u issues the copy of stream u of the stage (one
     // thread issuing every copy in turn is itself the bottleneck: each issue is a dependent
-    // chain of about a hundred cycles).
+    // chain of about a hundred cycles). Lane 0 also draws the CTA's next chunk from the step's
+    // counter and passes it to the consumers through a small queue in shared memory.
     const uint64_t pol = policy_evict_first();
-    uint32_t stage = 0, phase = 0, ss = 0, sphase = 0;
+    uint32_t stage = 0, phase = 0, ss = 0, sphase = 0, qi = 0, qphase = 0;
     uint32_t armed_g = 0, par_g = 0, armed_s = 0, par_s = 0;   // stages armed, and the parity of the last arming
     bool ok = true;
-    for (int c = c_begin; c < c_end && ok; ++c) {
-      const int t0 = A.chunk_tile0[c], nt = A.chunk_ntiles[c];
+    if (blockIdx.x == 0 && lane == 0) *A.next_chunk_reset = 0u;   // nobody reads it before the next step
+    // Lane 0 keeps the schedule two chunks deep, so that neither the draw (an atomic's round trip)
+    // nor the descriptor loads that depend on it are waited for: `cur` is the chunk being
+    // issued (descriptor in registers), `nxt` the index drawn one chunk ago, whose descriptor
+    // is requested now; the draw issued now is used one chunk later. The first chunk of CTA b
+    // is chunk b; draws hand out the chunks from `gridDim.x` on.
+    int cur = -1, c_t0 = 0, c_nt = 0, c_stride = 0, c_slot0 = 0;
+    unsigned nxt = 0u;
+    if (lane == 0) {
+      nxt = atomicAdd(A.next_chunk, 1u) + gridDim.x;
+      if ((int)blockIdx.x < A.nchunks) {
+        cur = (int)blockIdx.x;
+        c_t0 = A.chunk_tile0[cur]; c_nt = A.chunk_ntiles[cur]; c_stride = A.chunk_stride[cur]; c_slot0 = A.chunk_slot0[cur];
+      }
+    }
+    while (ok) {
+      ok = __all_sync(0xffffffffu, mbar_wait(empty_q + 8 * qi, qphase ^ 1u, give_up, A.err));
+      if (!ok) break;
+      int n_c = -1, n_t0 = 0, n_nt = 0, n_stride = 0, n_slot0 = 0;
+      unsigned drawn = 0u;
+      if (lane == 0) {
+        volatile int* e = queue + 8 * qi;
+        e[0] = cur; e[1] = c_t0; e[2] = c_nt; e[3] = c_stride; e[4] = c_slot0;
+        mbar_arrive(full_q + 8 * qi);                            // (release: the consumers' wait sees the entry)
+        if (cur >= 0) {
+          drawn = atomicAdd(A.next_chunk, 1u) + gridDim.x;
+          if (nxt < (unsigned)A.nchunks) {
+            n_c = (int)nxt;
+            n_t0 = A.chunk_tile0[n_c]; n_nt = A.chunk_ntiles[n_c]; n_stride = A.chunk_stride[n_c]; n_slot0 = A.chunk_slot0[n_c];
+          }
+        }
+      }
+      const int c = __shfl_sync(0xffffffffu, cur, 0);
+      if (++qi == QN) { qi = 0; qphase ^= 1u; }
+      if (c < 0) break;                                          // the list is exhausted: the consumers leave too
+      const int t0 = __shfl_sync(0xffffffffu, c_t0, 0), nt = __shfl_sync(0xffffffffu, c_nt, 0);
+      const int cstride = __shfl_sync(0xffffffffu, c_stride, 0);
       for (int i = 0; i < nt && ok; ++i) {
-        const int64_t tile_begin = (int64_t)tile_of(A, t0, i) * T;
+        const int64_t tile_begin = (int64_t)tile_of(A, t0, cstride, i) * T;
         if (tile_begin + T > A.P) break;  // the ragged last tile is read with plain loads
         for (int k0 = 0; k0 < A.K; k0 += G) {
           ok = __all_sync(0xffffffffu, mbar_wait(empty_g + 8 * stage, phase ^ 1u, give_up, A.err));
@@ -723,6 +812,8 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
         }
         if (++ss == NSS) { ss = 0; sphase ^= 1u; }
       }
+      cur = n_c; c_t0 = n_t0; c_nt = n_nt; c_stride = n_stride; c_slot0 = n_slot0;
+      nxt = drawn;
     }
     if (!ok && lane == 0) {
       // gave up: let the copies already issued land before the CTA's shared memory is released
@@ -742,14 +833,25 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
   const int tid = threadIdx.x;  // 0 .. CT-1
   Acc<KT, VEC> a;
   a.reset_chunk();
-  uint32_t stage = 0, phase = 0, ss = 0, sphase = 0;
+  MbarSync sy;
+  sy.bar = csync; sy.phase = 0u; sy.give_up = give_up; sy.err = A.err; sy.lane = lane;
+  uint32_t stage = 0, phase = 0, ss = 0, sphase = 0, qi = 0, qphase = 0;
   bool ok = true;
-  for (int c = c_begin; c < c_end; ++c) {
-    const int t0 = A.chunk_tile0[c], nt = A.chunk_ntiles[c];
-    float2* chunk_slots = A.slots + A.chunk_slot0[c];
-    SegState st; st.cur = -1; st.nent = 0; st.nbuf = 0;
+  SegState st; st.par = 0;
+  for (;;) {
+    // next chunk of this CTA, as drawn by the producer; a failed wait ends the CTA's work
+    ok = mbar_wait(full_q + 8 * qi, qphase, give_up, A.err) && ok;
+    volatile int* qe = queue + 8 * qi;
+    const int c = ok ? qe[0] : -1;
+    const int t0 = qe[1], nt = qe[2], cstride = qe[3], slot0 = qe[4];
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty_q + 8 * qi);
+    if (++qi == QN) { qi = 0; qphase ^= 1u; }
+    if (c < 0) break;
+    float2* chunk_slots = A.slots + slot0;
+    st.begin_chunk();
     for (int i = 0; i < nt; ++i) {
-      const int t = tile_of(A, t0, i);
+      const int t = tile_of(A, t0, cstride, i);
       const int tseg = A.tile_seg[t];          // needed only at the end of the tile: latency hidden
       const int64_t tile_begin = (int64_t)t * T;
       const int64_t jt = tile_begin + (int64_t)tid * VEC;
@@ -813,9 +915,9 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
 #pragma unroll
         for (int e = 0; e < VEC; ++e) { dv[e] = dv2[e]; nv[e] = nv2[e]; }
       }
-      segment_accumulate<KT, VEC, CW>(a, A, dv, nv, jt, tile_begin, tile_end, tseg, R, st, chunk_slots, 1, wid, lane);
+      segment_accumulate<KT, VEC, CW>(a, A, dv, nv, jt, tile_begin, tile_end, tseg, R, st, chunk_slots, sy, wid, lane);
     }
-    flush_chunk<KT, VEC, CW, ADAM>(a, A, R, st, c, chunk_slots, 1, wid, lane);
+    flush_chunk<KT, VEC, CW, ADAM>(a, A, R, st, c, chunk_slots, sy, wid, lane);
   }
 }
 
