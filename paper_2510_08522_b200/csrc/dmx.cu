@@ -244,16 +244,17 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
     }
   }
   std::vector<int32_t> chunk_tile0, chunk_ntiles, chunk_stride, chunk_slot0;
+  size_t last_tile_chunk = 0;                                   // the chunk that holds the last tile
   // smallest chunk: about 192 KB of streamed bytes (a few microseconds of one SM), so that the
   // per-chunk work (the draw, the reduction flush) stays small beside it
   const int64_t group_bytes = (int64_t)R * plan.tile * ((int64_t)K * (grad_dtype == DMX_BF16 ? 2 : 4) + 24);
   const int64_t min_groups = std::min<int64_t>(chunk_groups, std::max<int64_t>(1, (192 * 1024 + group_bytes - 1) / group_bytes));
   for (int64_t g0 = 0; g0 < ngroups;) {
     const int64_t rem = ngroups - g0;
-    const int64_t ng = rem <= 2 * min_groups * (int64_t)grid
-                           ? (rem + grid - 1) / grid      // the last wave: what is left, split evenly
-                           : std::max<int64_t>(min_groups, std::min<int64_t>(chunk_groups, rem / (2 * (int64_t)grid)));
-    const int64_t nl = std::min<int64_t>(grid, (rem + ng - 1) / ng);
+    const bool last_wave = rem <= 2 * min_groups * (int64_t)grid;   // what is left is split evenly over the CTAs
+    const int64_t ng = last_wave ? (rem + grid - 1) / grid
+                                 : std::max<int64_t>(min_groups, std::min<int64_t>(chunk_groups, rem / (2 * (int64_t)grid)));
+    const int64_t nl = last_wave ? std::min<int64_t>(grid, rem) : std::min<int64_t>(grid, (rem + ng - 1) / ng);
     const int64_t wave = std::min<int64_t>(rem, nl * ng);      // groups g0 .. g0+wave-1, lane l takes g0+l, g0+l+nl, ...
     for (int64_t l = 0; l < nl; ++l) {
       const int64_t n_l = (wave - l + nl - 1) / nl;
@@ -261,16 +262,17 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
       chunk_tile0.push_back((int32_t)((g0 + l) * R));
       chunk_ntiles.push_back((int32_t)((n_l - 1) * R + std::min<int64_t>(R, ntiles - glast * R)));
       chunk_stride.push_back((int32_t)(nl * R));
+      if (glast == ngroups - 1) last_tile_chunk = chunk_tile0.size() - 1;
     }
     g0 += wave;
   }
-  // The chunk that ends the list holds the last tile. If that tile is ragged it goes through the
-  // guarded plain-load path, several times slower than a full tile: drawn last it would extend
-  // the kernel by that much (8 % at P = 25.6 M), so it is drawn first instead.
-  if (P % plan.tile != 0 && chunk_tile0.size() > 1) {
-    std::rotate(chunk_tile0.begin(), chunk_tile0.end() - 1, chunk_tile0.end());
-    std::rotate(chunk_ntiles.begin(), chunk_ntiles.end() - 1, chunk_ntiles.end());
-    std::rotate(chunk_stride.begin(), chunk_stride.end() - 1, chunk_stride.end());
+  // If the last tile is ragged it goes through the guarded plain-load path, several times slower
+  // than a full tile: drawn near the end it would extend the kernel by that much (8 % at
+  // P = 25.6 M), so its chunk is moved to the front of the list, where CTA 0 starts with it.
+  if (P % plan.tile != 0 && last_tile_chunk > 0) {
+    std::rotate(chunk_tile0.begin(), chunk_tile0.begin() + last_tile_chunk, chunk_tile0.begin() + last_tile_chunk + 1);
+    std::rotate(chunk_ntiles.begin(), chunk_ntiles.begin() + last_tile_chunk, chunk_ntiles.begin() + last_tile_chunk + 1);
+    std::rotate(chunk_stride.begin(), chunk_stride.begin() + last_tile_chunk, chunk_stride.begin() + last_tile_chunk + 1);
   }
   const int nchunks = (int)chunk_tile0.size();
   // Enumerate, with the kernel's own rules, the (V, N) entries every chunk emits: a new entry

@@ -388,16 +388,21 @@ __device__ __forceinline__ void direct_tile(Acc<KT, Elem<BF16>::VEC>& a, const S
         if (k0 + u < KT && k0 + u < A.K) {
           const GT* src = static_cast<const GT*>(A.grad[k0 + u]) + jt;
           if constexpr (GUARD) {
-            uint32_t bits[VEC];
+            if (jt + VEC <= A.P) {              // the whole 16-byte piece is inside: one vector load
+              const uint4 r = ld_stream(src);
+              unpack2<BF16>(r, x[u]);
+            } else {                            // the piece that straddles P (and those beyond it): element by element
+              uint32_t bits[VEC];
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) {
-              bits[e] = 0u;
-              if (jt + e < A.P) {
-                if constexpr (BF16) bits[e] = (uint32_t)src[e] << 16; else bits[e] = __float_as_uint(src[e]);
+              for (int e = 0; e < VEC; ++e) {
+                bits[e] = 0u;
+                if (jt + e < A.P) {
+                  if constexpr (BF16) bits[e] = (uint32_t)src[e] << 16; else bits[e] = __float_as_uint(src[e]);
+                }
               }
-            }
 #pragma unroll
-            for (int i = 0; i < VEC / 2; ++i) x[u][i] = pk(bits[2 * i], bits[2 * i + 1]);
+              for (int i = 0; i < VEC / 2; ++i) x[u][i] = pk(bits[2 * i], bits[2 * i + 1]);
+            }
           } else {
             const uint4 r = ld_stream(src);
             unpack2<BF16>(r, x[u]);
@@ -747,43 +752,33 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
     uint32_t armed_g = 0, par_g = 0, armed_s = 0, par_s = 0;   // stages armed, and the parity of the last arming
     bool ok = true;
     if (blockIdx.x == 0 && lane == 0) *A.next_chunk_reset = 0u;   // nobody reads it before the next step
-    // Lane 0 keeps the schedule two chunks deep, so that neither the draw (an atomic's round trip)
-    // nor the descriptor loads that depend on it are waited for: `cur` is the chunk being
-    // issued (descriptor in registers), `nxt` the index drawn one chunk ago, whose descriptor
-    // is requested now; the draw issued now is used one chunk later. The first chunk of CTA b
-    // is chunk b; draws hand out the chunks from `gridDim.x` on.
+    // Lane 0 draws the next chunk a few tiles before the current chunk's copies have all been
+    // issued, and fetches its descriptor when they have (the ring then holds several
+    // microseconds of work, which covers that load). Drawing earlier would reserve chunks that a
+    // slow SM cannot start for a long time, which is what the dynamic schedule is there to avoid. The first chunk of CTA b is chunk b; draws
+    // hand out the chunks from `gridDim.x` on.
     int cur = -1, c_t0 = 0, c_nt = 0, c_stride = 0, c_slot0 = 0;
-    unsigned nxt = 0u;
-    if (lane == 0) {
-      nxt = atomicAdd(A.next_chunk, 1u) + gridDim.x;
-      if ((int)blockIdx.x < A.nchunks) {
-        cur = (int)blockIdx.x;
-        c_t0 = A.chunk_tile0[cur]; c_nt = A.chunk_ntiles[cur]; c_stride = A.chunk_stride[cur]; c_slot0 = A.chunk_slot0[cur];
-      }
+    if (lane == 0 && (int)blockIdx.x < A.nchunks) {
+      cur = (int)blockIdx.x;
+      c_t0 = A.chunk_tile0[cur]; c_nt = A.chunk_ntiles[cur]; c_stride = A.chunk_stride[cur]; c_slot0 = A.chunk_slot0[cur];
     }
     while (ok) {
       ok = __all_sync(0xffffffffu, mbar_wait(empty_q + 8 * qi, qphase ^ 1u, give_up, A.err));
       if (!ok) break;
-      int n_c = -1, n_t0 = 0, n_nt = 0, n_stride = 0, n_slot0 = 0;
       unsigned drawn = 0u;
       if (lane == 0) {
         volatile int* e = queue + 8 * qi;
         e[0] = cur; e[1] = c_t0; e[2] = c_nt; e[3] = c_stride; e[4] = c_slot0;
         mbar_arrive(full_q + 8 * qi);                            // (release: the consumers' wait sees the entry)
-        if (cur >= 0) {
-          drawn = atomicAdd(A.next_chunk, 1u) + gridDim.x;
-          if (nxt < (unsigned)A.nchunks) {
-            n_c = (int)nxt;
-            n_t0 = A.chunk_tile0[n_c]; n_nt = A.chunk_ntiles[n_c]; n_stride = A.chunk_stride[n_c]; n_slot0 = A.chunk_slot0[n_c];
-          }
-        }
       }
       const int c = __shfl_sync(0xffffffffu, cur, 0);
       if (++qi == QN) { qi = 0; qphase ^= 1u; }
       if (c < 0) break;                                          // the list is exhausted: the consumers leave too
       const int t0 = __shfl_sync(0xffffffffu, c_t0, 0), nt = __shfl_sync(0xffffffffu, c_nt, 0);
       const int cstride = __shfl_sync(0xffffffffu, c_stride, 0);
+      const int draw_at = nt > 3 ? nt - 3 : 0;
       for (int i = 0; i < nt && ok; ++i) {
+        if (lane == 0 && i == draw_at) drawn = atomicAdd(A.next_chunk, 1u) + gridDim.x;
         const int64_t tile_begin = (int64_t)tile_of(A, t0, cstride, i) * T;
         if (tile_begin + T > A.P) break;  // the ragged last tile is read with plain loads
         for (int k0 = 0; k0 < A.K; k0 += G) {
@@ -812,8 +807,13 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
         }
         if (++ss == NSS) { ss = 0; sphase ^= 1u; }
       }
-      cur = n_c; c_t0 = n_t0; c_nt = n_nt; c_stride = n_stride; c_slot0 = n_slot0;
-      nxt = drawn;
+      if (lane == 0) {
+        cur = -1;
+        if (drawn < (unsigned)A.nchunks) {
+          cur = (int)drawn;
+          c_t0 = A.chunk_tile0[cur]; c_nt = A.chunk_ntiles[cur]; c_stride = A.chunk_stride[cur]; c_slot0 = A.chunk_slot0[cur];
+        }
+      }
     }
     if (!ok && lane == 0) {
       // gave up: let the copies already issued land before the CTA's shared memory is released
