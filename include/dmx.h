@@ -189,6 +189,25 @@ int dmx_get_profile(dmx_handle* h, float* fused_ms, float* finalize_ms);
 int dmx_launches_per_step(const dmx_handle* h);
 
 /*
+ * dmx_plan_chunks — the work list dmx_create builds for the fused pass (host only: no CUDA call,
+ * no device needed). For inspection and for tests of the planning logic.
+ * The P parameters are cut into tiles of tile_elems elements (the last may be ragged); tiles are
+ * taken in groups of *group_tiles consecutive tiles; chunk c consists of num_tiles[c] tiles:
+ * tile i of the chunk is first_tile[c] + (i / G) * group_stride[c] + i % G with G = *group_tiles.
+ * Every tile belongs to exactly one chunk. The fused kernel's CTAs draw chunks in list order
+ * (CTA b starts with chunk b), so the list's order is the schedule: full waves first, shrinking
+ * waves towards the end, and the chunk holding a ragged last tile moved to the front.
+ *   resident_ctas   CTAs the device runs at once (SM count x CTAs per SM); *grid receives the
+ *                   number of CTAs the kernel is launched with
+ *   first_tile, num_tiles, group_stride   HOST, capacity entries each (may be NULL with capacity 0)
+ * Returns the number of chunks (the arrays are filled only if capacity is at least that), or
+ * DMX_ERR_ARG.
+ */
+int dmx_plan_chunks(int64_t P, int K, int grad_dtype, int tile_elems, int resident_ctas,
+                    int32_t* first_tile, int32_t* num_tiles, int32_t* group_stride, int capacity,
+                    int* group_tiles, int* grid);
+
+/*
  * Window statistics of the state vector over k consecutive steps, kept on the device.
  * The controller acts on metrics aggregated over k iterations (Section "System architecture";
  * Section "State representation": state vectors are built from metrics collected every k

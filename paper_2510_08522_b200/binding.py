@@ -21,7 +21,7 @@ FLAG_NONFINITE, FLAG_G2_NONPOS, FLAG_COS_UNDEF, FLAG_SINGLE, FLAG_INTERNAL = 1, 
 
 EXPORTS = ("dmx_create", "dmx_state_len", "dmx_step", "dmx_step_adam", "dmx_step_host", "dmx_step_static", "dmx_set_profiling", "dmx_get_profile",
            "dmx_launches_per_step", "dmx_destroy", "dmx_strerror", "dmx_last_cuda_error", "dmx_agg_create",
-           "dmx_agg_push", "dmx_agg_destroy", "dmx_ctl_num_features", "dmx_ctl_num_weights", "dmx_ctl_decide")
+           "dmx_agg_push", "dmx_agg_destroy", "dmx_ctl_num_features", "dmx_ctl_num_weights", "dmx_ctl_decide", "dmx_plan_chunks")
 CTL_ACTIONS = (-100, -25, 0, 25, 100)
 
 _lib = None
@@ -67,6 +67,8 @@ def lib():
         L.dmx_ctl_decide.argtypes = [i32, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, f32, f32, f32, f32, i32, i32,
                                      vp, vp, vp, vp, vp, vp, vp]
         L.dmx_ctl_decide.restype = i32
+        L.dmx_plan_chunks.argtypes = [i64, i32, i32, i32, i32, vp, vp, vp, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.dmx_plan_chunks.restype = i32
         L.dmx_set_profiling.argtypes = [vp, i32]
         L.dmx_set_profiling.restype = i32
         L.dmx_get_profile.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(f32)]
@@ -210,6 +212,20 @@ def ctl_decide(K, M, H, state_len, window, aux, batch, weights, cols=(-1, -1, -1
     if rc != OK:
         raise DmxError(rc, "dmx_ctl_decide")
     return out
+
+
+def dmx_plan_chunks(P, K, grad_dtype, tile_elems, resident_ctas):
+    """-> (code_or_count, first_tile, num_tiles, group_stride, group_tiles, grid): the fused pass's work
+    list as dmx_create would build it (host only; lists of ints)."""
+    R, G = ctypes.c_int(0), ctypes.c_int(0)
+    n = lib().dmx_plan_chunks(int(P), int(K), int(grad_dtype), int(tile_elems), int(resident_ctas), None, None, None, 0,
+                              ctypes.byref(R), ctypes.byref(G))
+    if n < 0:
+        return n, [], [], [], 0, 0
+    a, b, c = (ctypes.c_int32 * n)(), (ctypes.c_int32 * n)(), (ctypes.c_int32 * n)()
+    n = lib().dmx_plan_chunks(int(P), int(K), int(grad_dtype), int(tile_elems), int(resident_ctas), a, b, c, n,
+                              ctypes.byref(R), ctypes.byref(G))
+    return n, list(a), list(b), list(c), R.value, G.value
 
 
 def dmx_set_profiling(h, on) -> int:

@@ -148,6 +148,68 @@ Plan pick_pipe(int K) {
   return pipe_plan<64, BF16>();
 }
 
+// The chunk list of a problem: a function of (P, K, dtype, tile, resident CTAs, knobs) only.
+//
+// Tiles are taken in groups of R consecutive tiles; a chunk is a few groups, interleaved with
+// the other chunks of its wave: chunk l of a wave of n chunks that starts at group g0 holds
+// groups g0+l, g0+l+n, ... A full wave has one chunk per CTA. Chunks are about a sixth of a
+// CTA's share, at most 32 tiles (so that fp32 per-thread partials stay short) and at least 8:
+// SM speeds drift during a kernel, and on the mid-sized workloads 16-tile chunks measured 3-4 %
+// faster than 32-tile ones, while below 8 tiles the per-chunk work shows. Once fewer than two
+// such waves remain, every wave takes about half of what is left, down to a minimum chunk, so
+// that the CTAs finish together under the dynamic schedule. A chunk's sums do not depend on the
+// CTA that computes it, so results are reproducible on a given device.
+// Groups of 4 tiles measured 0.5-1 % faster than single tiles on the large workloads, groups of
+// 2 about 1 % faster on the mid-sized ones.
+struct ChunkPlan {
+  int R = 1, grid = 1;
+  std::vector<int32_t> tile0, ntiles, stride;   // per chunk: first tile, tiles, tiles between group starts
+};
+
+void plan_chunks(int64_t P, int K, int grad_dtype, int tile, int64_t sm_ctas, int want_R, int want_chunk, ChunkPlan& cp) {
+  const int64_t ntiles = (P + tile - 1) / tile;
+  const int auto_R = ntiles >= 4 * 64 * sm_ctas ? 4 : (ntiles >= 32 * sm_ctas ? 2 : 1);
+  const int R = std::max(1, std::min(want_R > 0 ? want_R : auto_R, 1 << 16));          // tiles per group
+  const int64_t share = (ntiles + sm_ctas - 1) / sm_ctas;                              // tiles per CTA
+  const int auto_chunk = (int)std::max<int64_t>(8, std::min<int64_t>(32, share / 6));
+  const int chunk_groups = std::max(1, (want_chunk > 0 ? want_chunk : auto_chunk) / R);
+  const int64_t ngroups = (ntiles + R - 1) / R;
+  const int grid = (int)std::min<int64_t>(sm_ctas, ngroups);
+  cp.R = R;
+  cp.grid = grid;
+  cp.tile0.clear(); cp.ntiles.clear(); cp.stride.clear();
+  size_t last_tile_chunk = 0;                                   // the chunk that holds the last tile
+  // smallest chunk: about 192 KB of streamed bytes (a few microseconds of one SM), so that the
+  // per-chunk work (the draw, the reduction flush) stays small beside it
+  const int64_t group_bytes = (int64_t)R * tile * ((int64_t)K * (grad_dtype == DMX_BF16 ? 2 : 4) + 24);
+  const int64_t min_groups = std::min<int64_t>(chunk_groups, std::max<int64_t>(1, (192 * 1024 + group_bytes - 1) / group_bytes));
+  for (int64_t g0 = 0; g0 < ngroups;) {
+    const int64_t rem = ngroups - g0;
+    // a problem of less than two minimum chunks per CTA is one wave, split evenly (nothing to balance)
+    const bool single = g0 == 0 && rem <= 2 * min_groups * (int64_t)grid;
+    const int64_t ng = single ? (rem + grid - 1) / grid
+                              : std::max<int64_t>(min_groups, std::min<int64_t>(chunk_groups, rem / (2 * (int64_t)grid)));
+    const int64_t nl = single ? std::min<int64_t>(grid, rem) : std::min<int64_t>(grid, (rem + ng - 1) / ng);
+    const int64_t wave = std::min<int64_t>(rem, nl * ng);      // groups g0 .. g0+wave-1, lane l takes g0+l, g0+l+nl, ...
+    for (int64_t l = 0; l < nl; ++l) {
+      const int64_t n_l = (wave - l + nl - 1) / nl;
+      const int64_t glast = g0 + l + (n_l - 1) * nl;            // only the very last group may be cut short by ntiles
+      cp.tile0.push_back((int32_t)((g0 + l) * R));
+      cp.ntiles.push_back((int32_t)((n_l - 1) * R + std::min<int64_t>(R, ntiles - glast * R)));
+      cp.stride.push_back((int32_t)(nl * R));
+      if (glast == ngroups - 1) last_tile_chunk = cp.tile0.size() - 1;
+    }
+    g0 += wave;
+  }
+  // If the last tile is ragged it goes through the guarded plain-load path, several times slower
+  // than a full tile: drawn near the end it would extend the kernel by that much (8 % at
+  // P = 25.6 M), so its chunk is moved to the front of the list, where CTA 0 starts with it.
+  if (P % tile != 0 && last_tile_chunk > 0) {
+    for (std::vector<int32_t>* v : {&cp.tile0, &cp.ntiles, &cp.stride})
+      std::rotate(v->begin(), v->begin() + last_tile_chunk, v->begin() + last_tile_chunk + 1);
+  }
+}
+
 void free_handle(dmx_handle* h) {
   if (!h) return;
   cudaFree(h->seg_off); cudaFree(h->tile_seg); cudaFree(h->chunk_stride); cudaFree(h->chunk_tile0);
@@ -210,29 +272,13 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   const int want = env_int("DMX_CTAS_PER_SM", 0);   // tuning knob: resident CTAs per SM (0 = all that fit)
   if (want > 0 && want < occ) occ = want;
   const int64_t ntiles = (P + plan.tile - 1) / plan.tile;
-  // Tiles are taken in groups of R consecutive tiles; a chunk is a few groups, interleaved with
-  // the other chunks of its wave: chunk l of a wave of n chunks that starts at group g0 holds
-  // groups g0+l, g0+l+n, ... A full wave has one chunk per CTA. Chunks are about a sixth of a
-  // CTA's share, at most `DMX_CHUNK_TILES` tiles (so that fp32 per-thread partials stay short) and
-  // at least 8: SM speeds drift during a kernel, and on the mid-sized workloads 16-tile chunks
-  // measured 3-4 % faster than 32-tile ones, while below 8 tiles the per-chunk work shows. Once
-  // fewer than two such waves remain, every wave takes about half of what is left, down to a
-  // minimum chunk, and the last wave splits its rest evenly, so that the CTAs finish together
-  // under the dynamic schedule. The list is a function of (P, tile, grid, R) only and a chunk's
-  // sums do not depend on the CTA that computes it: results are reproducible on a given device.
-  // Groups of 4 tiles measured 0.5-1 % faster than single tiles on the large workloads, groups
-  // of 2 about 1 % faster on the mid-sized ones.
   const int64_t sm_ctas = (int64_t)prop.multiProcessorCount * occ;
-  const int auto_R = ntiles >= 4 * 64 * sm_ctas ? 4 : (ntiles >= 32 * sm_ctas ? 2 : 1);
-  const int R = std::max(1, std::min(env_int("DMX_TILE_GROUP", auto_R), 1 << 16));   // tuning knob: tiles per group
-  const int64_t share = (ntiles + sm_ctas - 1) / sm_ctas;                            // tiles per CTA
-  const int auto_chunk = (int)std::max<int64_t>(8, std::min<int64_t>(32, share / 6));
-  const int chunk_groups = std::max(1, env_int("DMX_CHUNK_TILES", auto_chunk) / R);
-  const int64_t ngroups = (ntiles + R - 1) / R;
-  plan.grid = (int)std::min<int64_t>((int64_t)prop.multiProcessorCount * occ, ngroups);
+  ChunkPlan cp;
+  plan_chunks(P, K, grad_dtype, plan.tile, sm_ctas, env_int("DMX_TILE_GROUP", 0), env_int("DMX_CHUNK_TILES", 0), cp);
+  const int R = cp.R;
+  plan.grid = cp.grid;
   h->plan = plan;
   h->tile_group = R;
-  const int grid = plan.grid;
   // per-tile segment table
   std::vector<int32_t> tile_seg((size_t)ntiles);
   {
@@ -243,37 +289,8 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
       tile_seg[(size_t)t] = s | (seg_offsets[s + 1] < j1 && s < S - 1 ? dmx::kTileBoundaryBit : 0);
     }
   }
-  std::vector<int32_t> chunk_tile0, chunk_ntiles, chunk_stride, chunk_slot0;
-  size_t last_tile_chunk = 0;                                   // the chunk that holds the last tile
-  // smallest chunk: about 192 KB of streamed bytes (a few microseconds of one SM), so that the
-  // per-chunk work (the draw, the reduction flush) stays small beside it
-  const int64_t group_bytes = (int64_t)R * plan.tile * ((int64_t)K * (grad_dtype == DMX_BF16 ? 2 : 4) + 24);
-  const int64_t min_groups = std::min<int64_t>(chunk_groups, std::max<int64_t>(1, (192 * 1024 + group_bytes - 1) / group_bytes));
-  for (int64_t g0 = 0; g0 < ngroups;) {
-    const int64_t rem = ngroups - g0;
-    const bool last_wave = rem <= 2 * min_groups * (int64_t)grid;   // what is left is split evenly over the CTAs
-    const int64_t ng = last_wave ? (rem + grid - 1) / grid
-                                 : std::max<int64_t>(min_groups, std::min<int64_t>(chunk_groups, rem / (2 * (int64_t)grid)));
-    const int64_t nl = last_wave ? std::min<int64_t>(grid, rem) : std::min<int64_t>(grid, (rem + ng - 1) / ng);
-    const int64_t wave = std::min<int64_t>(rem, nl * ng);      // groups g0 .. g0+wave-1, lane l takes g0+l, g0+l+nl, ...
-    for (int64_t l = 0; l < nl; ++l) {
-      const int64_t n_l = (wave - l + nl - 1) / nl;
-      const int64_t glast = g0 + l + (n_l - 1) * nl;            // only the very last group may be cut short by ntiles
-      chunk_tile0.push_back((int32_t)((g0 + l) * R));
-      chunk_ntiles.push_back((int32_t)((n_l - 1) * R + std::min<int64_t>(R, ntiles - glast * R)));
-      chunk_stride.push_back((int32_t)(nl * R));
-      if (glast == ngroups - 1) last_tile_chunk = chunk_tile0.size() - 1;
-    }
-    g0 += wave;
-  }
-  // If the last tile is ragged it goes through the guarded plain-load path, several times slower
-  // than a full tile: drawn near the end it would extend the kernel by that much (8 % at
-  // P = 25.6 M), so its chunk is moved to the front of the list, where CTA 0 starts with it.
-  if (P % plan.tile != 0 && last_tile_chunk > 0) {
-    std::rotate(chunk_tile0.begin(), chunk_tile0.begin() + last_tile_chunk, chunk_tile0.begin() + last_tile_chunk + 1);
-    std::rotate(chunk_ntiles.begin(), chunk_ntiles.begin() + last_tile_chunk, chunk_ntiles.begin() + last_tile_chunk + 1);
-    std::rotate(chunk_stride.begin(), chunk_stride.begin() + last_tile_chunk, chunk_stride.begin() + last_tile_chunk + 1);
-  }
+  std::vector<int32_t>&chunk_tile0 = cp.tile0, &chunk_ntiles = cp.ntiles, &chunk_stride = cp.stride;
+  std::vector<int32_t> chunk_slot0;
   const int nchunks = (int)chunk_tile0.size();
   // Enumerate, with the kernel's own rules, the (V, N) entries every chunk emits: a new entry
   // whenever the running segment changes between tiles, at every boundary crossed inside a
@@ -434,10 +451,23 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
   h->step_parity ^= 1u;   // only a step that was enqueued consumes its counter
   if (prof && !cuda_ok(cudaEventRecord(h->ev[1], stream))) return DMX_ERR_CUDA;
-  const int funits = K + 2 + 2 * F.adam + h->nunits;   // one warp per chunk-row column and per segment unit
-  const int fblocks = (funits + dmx::kFinalWarps - 1) / dmx::kFinalWarps;
-  dmx::finalize_kernel<<<fblocks, dmx::kFinalWarps * 32, 0, stream>>>(F);
-  if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
+  // one block per chunk-row column, one warp per segment unit. Launched as a programmatic
+  // dependent of the fused pass: its blocks may become resident while that kernel drains and
+  // wait (griddepcontrol.wait) for its completion, which hides the launch latency between the
+  // two kernels. With per-kernel timing on, the event between them needs the plain ordering.
+  const int fblocks = K + 2 + 2 * F.adam + (h->nunits + dmx::kFinalWarps - 1) / dmx::kFinalWarps;
+  cudaLaunchConfig_t cfg;
+  std::memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)fblocks);
+  cfg.blockDim = dim3(dmx::kFinalWarps * 32);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  std::memset(attr, 0, sizeof(attr));
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = prof ? 0 : 1;
+  if (!cuda_ok(cudaLaunchKernelEx(&cfg, dmx::finalize_kernel, F))) return DMX_ERR_CUDA;
   if (prof) {
     if (!cuda_ok(cudaEventRecord(h->ev[2], stream))) return DMX_ERR_CUDA;
     h->profiled = true;
@@ -502,6 +532,24 @@ int dmx_get_profile(dmx_handle* h, float* fused_ms, float* finalize_ms) {
   if (!cuda_ok(cudaEventElapsedTime(fused_ms, h->ev[0], h->ev[1]))) return DMX_ERR_CUDA;
   if (!cuda_ok(cudaEventElapsedTime(finalize_ms, h->ev[1], h->ev[2]))) return DMX_ERR_CUDA;
   return DMX_OK;
+}
+
+int dmx_plan_chunks(int64_t P, int K, int grad_dtype, int tile_elems, int resident_ctas, int32_t* first_tile,
+                    int32_t* num_tiles, int32_t* group_stride, int capacity, int* group_tiles, int* grid) {
+  if (P < 1 || P >= DMX_MAX_PARAMS || K < 1 || K > DMX_MAX_WORKERS || tile_elems < 1 || resident_ctas < 1 ||
+      (grad_dtype != DMX_F32 && grad_dtype != DMX_BF16) || capacity < 0)
+    return DMX_ERR_ARG;
+  ChunkPlan cp;
+  plan_chunks(P, K, grad_dtype, tile_elems, resident_ctas, 0, 0, cp);
+  if (group_tiles) *group_tiles = cp.R;
+  if (grid) *grid = cp.grid;
+  const int n = (int)cp.tile0.size();
+  if (capacity >= n && first_tile && num_tiles && group_stride) {
+    std::copy(cp.tile0.begin(), cp.tile0.end(), first_tile);
+    std::copy(cp.ntiles.begin(), cp.ntiles.end(), num_tiles);
+    std::copy(cp.stride.begin(), cp.stride.end(), group_stride);
+  }
+  return n;
 }
 
 int dmx_launches_per_step(const dmx_handle* h) {

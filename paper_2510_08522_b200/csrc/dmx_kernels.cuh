@@ -508,41 +508,59 @@ constexpr int kFinalWarps = 8;
 
 constexpr int kFinalPart = 256;  // slots per segment unit
 
-// First level: one warp per unit. Units 0..K+1 are the columns q_k, c, pp of the chunk rows;
-// the others are runs of at most kFinalPart slots of one segment. Second level, in the last
+// First level. Blocks 0..ncol-1 each sum one column (q_k, c, pp, and Adam's two) of the chunk
+// rows: warp w takes the w-th eighth of the column, lanes stride through it with eight loads in
+// flight, and the eight warp sums are added in warp order. The other blocks take segment units
+// (runs of at most kFinalPart slots of one segment), one warp each. Second level, in the last
 // block to finish: the units of each segment in order, then the derived scalars.
 static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const __grid_constant__ FinalArgs F) {
   const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int K = F.K, S = F.S;
-  const int unit = blockIdx.x * kFinalWarps + wid;
   const int ncol = K + 2 + 2 * F.adam;
-  if (unit < ncol) {
-    const float* col = F.rows + (int64_t)unit * F.nchunks;
-    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-    int c = lane;
-    for (; c + 96 < F.nchunks; c += 128) {
-      a0 += (double)col[c]; a1 += (double)col[c + 32]; a2 += (double)col[c + 64]; a3 += (double)col[c + 96];
+  __shared__ double s_col[kFinalWarps];
+  // everything this kernel reads was written by the step's fused pass: with a programmatic
+  // dependent launch this is where its completion (and the visibility of its writes) is awaited
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if ((int)blockIdx.x < ncol) {
+    const float* col = F.rows + (int64_t)blockIdx.x * F.nchunks;
+    const int per = (F.nchunks + kFinalWarps - 1) / kFinalWarps;
+    const int lo = wid * per, hi = lo + per < F.nchunks ? lo + per : F.nchunks;
+    double a[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a[i] = 0.0;
+    int c = lo + lane;
+    for (; c + 224 < hi; c += 256) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) a[i] += (double)col[c + 32 * i];
     }
-    for (; c < F.nchunks; c += 32) a0 += (double)col[c];
-    const double acc = warp_sum_d((a0 + a1) + (a2 + a3));
-    if (lane == 0) F.colsum[unit] = acc;
-  } else if (unit < ncol + F.nunits) {
-    const int u = unit - ncol;
-    const int lo = F.unit_lo[u], hi = F.unit_hi[u];
-    double v = 0.0, n = 0.0, v1 = 0.0, n1 = 0.0, v2 = 0.0, n2 = 0.0, v3 = 0.0, n3 = 0.0;
-    int i = lo + lane;
-    for (; i + 96 < hi; i += 128) {          // four gathers in flight per lane; fixed summation order
-      const int i0 = F.seg_slots[i], i1 = F.seg_slots[i + 32], i2 = F.seg_slots[i + 64], i3 = F.seg_slots[i + 96];
-      const float2 t0 = F.slots[i0], t1 = F.slots[i1], t2 = F.slots[i2], t3 = F.slots[i3];
-      v += (double)t0.x; n += (double)t0.y; v1 += (double)t1.x; n1 += (double)t1.y;
-      v2 += (double)t2.x; n2 += (double)t2.y; v3 += (double)t3.x; n3 += (double)t3.y;
+    for (; c < hi; c += 32) a[0] += (double)col[c];
+    const double acc = warp_sum_d(((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7])));
+    if (lane == 0) s_col[wid] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double t = 0.0;
+      for (int w = 0; w < kFinalWarps; ++w) t += s_col[w];
+      F.colsum[blockIdx.x] = t;
     }
-    for (; i < hi; i += 32) {
-      const float2 t = F.slots[F.seg_slots[i]];
-      v += (double)t.x; n += (double)t.y;
+  } else {
+    const int u = ((int)blockIdx.x - ncol) * kFinalWarps + wid;
+    if (u < F.nunits) {
+      const int lo = F.unit_lo[u], hi = F.unit_hi[u];
+      double v = 0.0, n = 0.0, v1 = 0.0, n1 = 0.0, v2 = 0.0, n2 = 0.0, v3 = 0.0, n3 = 0.0;
+      int i = lo + lane;
+      for (; i + 96 < hi; i += 128) {          // four gathers in flight per lane; fixed summation order
+        const int i0 = F.seg_slots[i], i1 = F.seg_slots[i + 32], i2 = F.seg_slots[i + 64], i3 = F.seg_slots[i + 96];
+        const float2 t0 = F.slots[i0], t1 = F.slots[i1], t2 = F.slots[i2], t3 = F.slots[i3];
+        v += (double)t0.x; n += (double)t0.y; v1 += (double)t1.x; n1 += (double)t1.y;
+        v2 += (double)t2.x; n2 += (double)t2.y; v3 += (double)t3.x; n3 += (double)t3.y;
+      }
+      for (; i < hi; i += 32) {
+        const float2 t = F.slots[F.seg_slots[i]];
+        v += (double)t.x; n += (double)t.y;
+      }
+      v = warp_sum_d((v + v1) + (v2 + v3)); n = warp_sum_d((n + n1) + (n2 + n3));
+      if (lane == 0) F.segpart[u] = make_double2(v, n);
     }
-    v = warp_sum_d((v + v1) + (v2 + v3)); n = warp_sum_d((n + n1) + (n2 + n3));
-    if (lane == 0) F.segpart[u] = make_double2(v, n);
   }
   __shared__ unsigned s_last;
   __shared__ double s_red[2][kFinalWarps];
@@ -738,6 +756,8 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
+  // the step's second kernel may be made resident from now on; it waits for this grid to complete
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   constexpr int ESZ = BF16 ? 2 : 4;
 
   if (wid == CW) {
