@@ -1,0 +1,103 @@
+"""More GPU cases through the C ABI: the plain-load kernel (DMX_KERNEL=direct) against the
+oracle, the scheduling knobs (results must not depend on them beyond rounding), and a problem
+of more than 2^32 elements checked by closed forms."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle.dmx_oracle import Oracle
+from paper_2510_08522_b200 import workload as W
+from tests import parity as PT
+from tests.test_gpu_parity import Custom, _dmx, _torch, free_run, rnd
+
+pytestmark = pytest.mark.gpu
+
+
+class env:
+    def __init__(self, **kv):
+        self.kv = kv
+
+    def __enter__(self):
+        self.old = {k: os.environ.get(k) for k in self.kv}
+        os.environ.update({k: str(v) for k, v in self.kv.items()})
+
+    def __exit__(self, *a):
+        for k, v in self.old.items():
+            if v is None:
+                os.environ.pop(k, None)
+            else:
+                os.environ[k] = v
+
+
+@pytest.mark.parametrize("idx,P,steps", [(0, 262_147, 2), (1, 333_337, 3), (2, 401_239, 3), (3, 290_011, 2), (4, 523_777, 2)])
+def test_plain_load_kernel_matches_oracle(idx, P, steps):
+    with env(DMX_KERNEL="direct"):
+        free_run(W.WORKLOADS[idx].scaled(P=P, steps=steps), steps)
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_plain_load_kernel_shapes(dtype):
+    with env(DMX_KERNEL="direct"):
+        for K, P, seg in [(1, 5, [0, 5]), (3, 2049, [0, 1, 1, 700, 2049]), (33, 20_011, [0, 9, 10_000, 20_011]),
+                          (64, 9_973, [0, 9_973])]:
+            Custom(rnd(K + P, K, P), [32 * (1 + k % 5) for k in range(K)], seg, dtype).run(what="direct K=%d P=%d" % (K, P))
+
+
+@pytest.mark.parametrize("knobs", [dict(DMX_TILE_GROUP=1, DMX_CHUNK_TILES=1), dict(DMX_TILE_GROUP=3, DMX_CHUNK_TILES=7),
+                                   dict(DMX_TILE_GROUP=8, DMX_CHUNK_TILES=64), dict(DMX_CTAS_PER_SM=1, DMX_CHUNK_TILES=4)])
+def test_scheduling_knobs_do_not_change_results_beyond_rounding(knobs):
+    # many chunks per CTA, odd group sizes, segment boundaries at every residue: the work list and
+    # the slot bookkeeping must stay consistent for any cut
+    K, P = 6, 1_300_003
+    seg = [0] + sorted(set(int(v) for v in np.random.default_rng(5).integers(1, P, 40))) + [P]
+    with env(**knobs):
+        for dtype in (0, 1):
+            Custom(rnd(17, K, P), [16, 48, 32, 256, 64, 1024], seg, dtype).run(what="knobs %r" % (knobs,))
+
+
+def test_more_than_2_to_32_elements_closed_forms():
+    """Index arithmetic beyond 32 bits. Two workers share one constant bf16 gradient buffer
+    (identical workers: g = x exactly, no spread), so every output has a closed form:
+    A = q_k = P c^2, m' = beta m + c, theta' = theta - lr m'; slices of the per-element
+    outputs are compared at the ends and around the 2^31 and 2^32 element marks."""
+    torch, D = _torch(), _dmx()
+    P = (1 << 32) + 1_234_567
+    free, _ = torch.cuda.mem_get_info()
+    if free < P * 14 + (4 << 30):
+        pytest.skip("needs about 64 GB of free device memory")
+    c = 0.0078125                                    # 2^-7: exact in bf16, P c^2 exact in fp64
+    g = torch.full((P,), c, dtype=torch.bfloat16, device="cuda")
+    gen = torch.Generator(device="cuda").manual_seed(1)
+    params = torch.empty(P, dtype=torch.float32, device="cuda").normal_(0, 0.05, generator=gen)
+    mom = torch.empty(P, dtype=torch.float32, device="cuda").normal_(0, 0.01, generator=gen)
+    prev = torch.full((P,), 2 * c, dtype=torch.float32, device="cuda")
+    seg = [0, 1 << 31, (1 << 32) - 3, (1 << 32) + 5, P]
+    marks = [0, (1 << 31) - 4096, (1 << 32) - 4096, P - 8192]
+    before = [(params[a:a + 8192].cpu().numpy().astype(np.float64), mom[a:a + 8192].cpu().numpy().astype(np.float64)) for a in marks]
+    sum_m0 = float(torch.sum(mom, dtype=torch.float64))
+    d = D.Dmx(2, P, seg, W.BF16)
+    lr, beta = np.float32(0.1), np.float32(0.9)
+    st = d.step([g, g], [32, 96], params, mom, float(lr), float(beta), prev)
+    torch.cuda.synchronize()
+    st = st.cpu().numpy().astype(np.float64)
+    d.close()
+    A = P * c * c
+    assert st[0] == 128 and st[11] == 0
+    assert abs(st[1] - A) <= 1e-4 * A and st[2] == 0.0 and abs(st[3] - A) <= 1e-4 * A and st[4] == 0.0
+    assert abs(st[5] - 1.0) <= 1e-4 and abs(st[6] - 2 * A) <= 2e-4 * A and abs(st[7] - 4 * A) <= 4e-4 * A
+    assert np.allclose(st[16:18], A, rtol=1e-4)
+    sizes = np.diff(np.array(seg, dtype=np.float64))
+    assert np.all(st[18:22] == 0.0) and np.allclose(st[22:26], sizes * c * c, rtol=1e-4)
+    for a, (p0, m0) in zip(marks, before):
+        m1 = float(beta) * m0 + c
+        p1 = p0 - float(lr) * m1
+        assert np.array_equal(prev[a:a + 8192].cpu().numpy(), np.full(8192, c, np.float32))
+        assert np.allclose(mom[a:a + 8192].cpu().numpy(), m1, rtol=1e-6, atol=1e-9)
+        assert np.allclose(params[a:a + 8192].cpu().numpy(), p1, rtol=1e-6, atol=1e-9)
+    # nothing outside the sampled slices was skipped or done twice: the updated momentum's total
+    # matches its closed form
+    sum_m1 = float(torch.sum(mom, dtype=torch.float64))
+    assert abs(sum_m1 - (float(beta) * sum_m0 + P * c)) <= 1e-6 * P * c
+    del g, params, prev, mom
+    torch.cuda.empty_cache()
