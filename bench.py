@@ -119,8 +119,13 @@ def step_bytes(wl, optimizer):
     return wl.bytes_per_step + (8 * wl.P if optimizer == "adam" else 0)
 
 
+L2_FLUSH_BELOW = 4 << 30      # workloads streaming less than this per step get an L2 flush between steps
+
+
 def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profile=True, optimizer="sgd"):
-    """Time `steps` steps of workload `wl` on `device`. Returns a dict of local measurements."""
+    """Time `steps` steps of workload `wl` on `device`. Returns a dict of local measurements.
+    Workloads whose step streams only a few times the L2's size get a 512 MB write between the
+    (untimed) input generation and the timed step, so that no step starts on a warm L2."""
     import torch
     import paper_2510_08522_b200 as D
     from paper_2510_08522_b200 import workload as W
@@ -131,6 +136,7 @@ def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profi
     out_state = torch.empty(d.state_len, dtype=torch.float32, device=device)
     d.set_profiling(profile)
     second = torch.zeros(wl.P, dtype=torch.float32, device=device) if optimizer == "adam" else None
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=device) if step_bytes(wl, optimizer) < L2_FLUSH_BELOW else None
     tcount = [0]
 
     def one_step(b):
@@ -153,6 +159,8 @@ def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profi
     wall0 = time.time()
     for s in range(steps):
         b = dp.fill()                     # untimed: next step's gradients
+        if flush is not None:
+            flush.zero_()                 # untimed: evicts the freshly written gradients and the state from L2
         ev[s][0].record()
         one_step(b)
         ev[s][1].record()
@@ -166,7 +174,8 @@ def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profi
     times = [e0.elapsed_time(e1) for e0, e1 in ev]
     flags = int(out_state[11].item())
     res = dict(total_ms=sum(times), times=times, fused_ms=fused, finalize_ms=fin, clocks=clocks, flags=flags,
-               wall_s=wall, launches=steps * d.launches_per_step)
+               wall_s=wall, launches=steps * d.launches_per_step, l2_flushed=flush is not None)
+    del flush
 
     # end to end: gradients start in pinned host memory, the state vector ends in host memory
     if e2e_steps > 0 and optimizer == "sgd":
@@ -246,6 +255,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=4, help="index into the workload table (default: the largest)")
     ap.add_argument("--also", type=int, default=3, help="second workload reported under 'also' (-1: none)")
+    ap.add_argument("--all-workloads", type=int, default=1,
+                    help="1: also time the remaining workloads briefly and list them under 'workloads' (N=1 only)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-sample-elems", type=int, default=128 << 20, help="0: skip the CPU-baseline leg")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "adam"],
@@ -265,7 +276,8 @@ def main():
     config = {"workload": wl.name, "K": wl.K, "P": wl.P, "S": wl.S,
               "grad_dtype": "bf16" if wl.dtype == W.BF16 else "f32", "optimizer": args.optimizer,
               "bytes_per_step": step_bytes(wl, args.optimizer),
-              "l2": "inputs larger than L2 (gradients regenerated between steps)", "parallelism": "replicas x%d" % args.gpus}
+              "l2": ("flushed between steps (512 MB write)" if step_bytes(wl, args.optimizer) < L2_FLUSH_BELOW
+                     else "inputs larger than L2 (gradients regenerated between steps)"), "parallelism": "replicas x%d" % args.gpus}
 
     if args.impl == "reference":
         if rank != 0:
@@ -319,6 +331,23 @@ def main():
                 "steps_per_s": 1e3 / ms2, "bytes_per_step": nb2,
                 "roofline_frac": nb2 / f2 / 1e6 / peak, "fused_kernel_ms": f2}
 
+    others = []
+    if args.all_workloads and world == 1 and not args.P:
+        peak_o, _ = measured_peak()
+        for i, wlo in enumerate(W.WORKLOADS):
+            if i in (args.workload, args.also):
+                continue
+            ro = run_workload(wlo, max(5, args.steps // 2), args.warmup, device, 0, sample_clocks=False, optimizer=args.optimizer)
+            del ro["problem"]
+            torch.cuda.empty_cache()
+            mso = ro["total_ms"] / len(ro["times"])
+            fo = sum(ro["fused_ms"]) / len(ro["fused_ms"])
+            nbo = step_bytes(wlo, args.optimizer)
+            others.append({"workload": wlo.name, "value": nbo / mso / 1e6, "unit": UNIT, "ms_per_step": mso,
+                           "steps_per_s": 1e3 / mso, "bytes_per_step": nbo, "fused_kernel_ms": fo,
+                           "roofline_frac": nbo / fo / 1e6 / peak_o,
+                           "l2": "flushed between steps" if ro["l2_flushed"] else "inputs larger than L2"})
+
     if rank != 0:
         DU.finish()
         return 0
@@ -349,6 +378,8 @@ def main():
                        "note": "gradients copied from pinned host memory every step; params, momentum and prev_agg stay resident"}
     if also:
         line["also"] = also
+    if others:
+        line["workloads"] = others
     if world == 1 and args.cpu_sample_elems > 0:
         ts, sub = oracle_sample(wl, args.cpu_sample_elems, ncores, reps=1, device=device)
         line["cpu_baseline"] = {"value": sub.bytes_per_step / ts[0] / 1e9, "unit": UNIT, "cores": ncores, "kind": "oracle",

@@ -158,6 +158,53 @@ int dmx_step_adam(dmx_handle* h, const void* const* grad_ptrs, const int32_t* ba
 enum { DMX_ST_ADAM_GHAT_MEAN = 12, DMX_ST_ADAM_GHAT_VAR = 13, DMX_ST_ADAM_GHAT_STD = 14 };
 
 /*
+ * Sharding one problem by parameter range (several GPUs, or several passes on one).
+ * Every output of the step is either per parameter or a sum over parameters, so a problem splits
+ * by parameter range with one small exchange: shard r owns elements [lo, hi) of all K gradient
+ * buffers and of params/momentum/prev_agg, runs the same fused pass on them, and emits its raw
+ * fp64 sums; the shards' sums are added (an all-reduce of K + 5 + 2 S doubles: the one exchange
+ * step, e.g. NCCL over NVLink), and the state vector is derived from the total. This mirrors
+ * the paper's scaling of the worker loop over 8 to 32 nodes (Section "Scalability of DYNAMIX"); the
+ * paper has no formula for it. In a cluster where worker k is GPU k, the gradient shards come from
+ * a reduce-scatter-like exchange that leaves every GPU with all workers' values of its range.
+ *
+ *   dmx_shard_range     HOST only. [lo, hi) of shard `shard` of `nshards`: boundaries on multiples
+ *                       of 1024 elements (pointer alignment survives), the last shard ends at P;
+ *                       a shard may be empty (lo == hi) when P is small: skip it.
+ *   dmx_shard_segments  HOST only. The shard's own segment table (S+1 entries, written to
+ *                       shard_offsets): the problem's table clipped to [lo, hi) and shifted by lo;
+ *                       segments outside the shard become empty. Create the shard's handle with
+ *                       dmx_create(K, hi - lo, shard_offsets, S, dtype): S and the state layout
+ *                       stay those of the whole problem.
+ *   dmx_partials_len    K + 5 + 2 S.
+ *   dmx_step_partial, dmx_step_adam_partial
+ *                       as dmx_step / dmx_step_adam on the shard's buffers (pointers to element lo),
+ *                       but instead of out_state they write `partials` (DEVICE, dmx_partials_len
+ *                       doubles, 8-byte aligned): q_k [K] in the caller's worker order, <g,a>, |a|^2,
+ *                       Adam's sum and sum of squares of ghat (0 for SGD), Vraw_s [S] (before the
+ *                       division by K-1), N_s [S], and a word that is non-zero if a bounded wait
+ *                       inside the kernel ran out.
+ *   dmx_finalize_partials
+ *                       batch_sizes: HOST, K ints; partials: DEVICE, the entry-wise sum over all
+ *                       shards; P_total: the whole problem's parameter count (Adam's mean); writes
+ *                       out_state (DEVICE, 16 + K + 2 S fp32) exactly as dmx_step defines it.
+ *                       Asynchronous, one small launch.
+ * Errors as dmx_step; DMX_ERR_SEGMENTS for a bad table or a range outside it.
+ */
+int dmx_shard_range(int64_t P, int nshards, int shard, int64_t* lo, int64_t* hi);
+int dmx_shard_segments(const int64_t* seg_offsets, int S, int64_t lo, int64_t hi, int64_t* shard_offsets);
+int dmx_partials_len(const dmx_handle* h);
+int dmx_step_partial(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes, float* params,
+                     float* momentum, float lr, float beta, float* prev_agg, double* partials,
+                     void* cuda_stream);
+int dmx_step_adam_partial(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes,
+                          float* params, float* first_moment, float* second_moment, float lr, float beta1,
+                          float beta2, float eps, int64_t t, float* prev_agg, double* partials,
+                          void* cuda_stream);
+int dmx_finalize_partials(int K, int S, const int32_t* batch_sizes, const double* partials, int adam,
+                          int64_t P_total, float* out_state, void* cuda_stream);
+
+/*
  * dmx_step_host — the same step for a caller whose gradients sit in HOST memory (the end-to-end
  * form of Algorithm 1's worker loop on one machine: gradients arrive from the workers' side of
  * the bus, the model state stays resident on the GPU).

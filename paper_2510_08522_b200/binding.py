@@ -21,7 +21,9 @@ FLAG_NONFINITE, FLAG_G2_NONPOS, FLAG_COS_UNDEF, FLAG_SINGLE, FLAG_INTERNAL = 1, 
 
 EXPORTS = ("dmx_create", "dmx_state_len", "dmx_step", "dmx_step_adam", "dmx_step_host", "dmx_step_static", "dmx_set_profiling", "dmx_get_profile",
            "dmx_launches_per_step", "dmx_destroy", "dmx_strerror", "dmx_last_cuda_error", "dmx_agg_create",
-           "dmx_agg_push", "dmx_agg_destroy", "dmx_ctl_num_features", "dmx_ctl_num_weights", "dmx_ctl_decide", "dmx_plan_chunks")
+           "dmx_agg_push", "dmx_agg_destroy", "dmx_ctl_num_features", "dmx_ctl_num_weights", "dmx_ctl_decide", "dmx_plan_chunks",
+           "dmx_shard_range", "dmx_shard_segments", "dmx_partials_len", "dmx_step_partial", "dmx_step_adam_partial",
+           "dmx_finalize_partials")
 CTL_ACTIONS = (-100, -25, 0, 25, 100)
 
 _lib = None
@@ -69,6 +71,18 @@ def lib():
         L.dmx_ctl_decide.restype = i32
         L.dmx_plan_chunks.argtypes = [i64, i32, i32, i32, i32, vp, vp, vp, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
         L.dmx_plan_chunks.restype = i32
+        L.dmx_shard_range.argtypes = [i64, i32, i32, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+        L.dmx_shard_range.restype = i32
+        L.dmx_shard_segments.argtypes = [vp, i32, i64, i64, vp]
+        L.dmx_shard_segments.restype = i32
+        L.dmx_partials_len.argtypes = [vp]
+        L.dmx_partials_len.restype = i32
+        L.dmx_step_partial.argtypes = [vp, vp, vp, vp, vp, f32, f32, vp, vp, vp]
+        L.dmx_step_partial.restype = i32
+        L.dmx_step_adam_partial.argtypes = [vp, vp, vp, vp, vp, vp, f32, f32, f32, f32, i64, vp, vp, vp]
+        L.dmx_step_adam_partial.restype = i32
+        L.dmx_finalize_partials.argtypes = [i32, i32, vp, vp, i32, i64, vp, vp]
+        L.dmx_finalize_partials.restype = i32
         L.dmx_set_profiling.argtypes = [vp, i32]
         L.dmx_set_profiling.restype = i32
         L.dmx_get_profile.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(f32)]
@@ -214,6 +228,53 @@ def ctl_decide(K, M, H, state_len, window, aux, batch, weights, cols=(-1, -1, -1
     return out
 
 
+def dmx_shard_range(P, nshards, shard):
+    """-> (code, lo, hi): the parameter range of one shard (host only)."""
+    lo, hi = ctypes.c_int64(0), ctypes.c_int64(0)
+    rc = lib().dmx_shard_range(int(P), int(nshards), int(shard), ctypes.byref(lo), ctypes.byref(hi))
+    return rc, lo.value, hi.value
+
+
+def dmx_shard_segments(seg_offsets, lo, hi):
+    """-> (code, shard_offsets): the problem's segment table clipped to [lo, hi) and shifted (host only)."""
+    n = len(seg_offsets)
+    seg = (ctypes.c_int64 * n)(*[int(v) for v in seg_offsets])
+    out = (ctypes.c_int64 * n)()
+    rc = lib().dmx_shard_segments(seg, n - 1, int(lo), int(hi), out)
+    return rc, list(out)
+
+
+def dmx_partials_len(h) -> int:
+    return lib().dmx_partials_len(h)
+
+
+def dmx_step_partial(h, grad_ptrs, batch_sizes, params, momentum, lr, beta, prev_agg, partials, stream=0) -> int:
+    """dmx_step on a parameter shard: raw fp64 sums to `partials` (device address) instead of a state vector."""
+    K = len(grad_ptrs)
+    gp = (ctypes.c_void_p * K)(*[int(p) for p in grad_ptrs])
+    bs = (ctypes.c_int32 * K)(*[int(b) for b in batch_sizes])
+    return lib().dmx_step_partial(h, gp, bs, int(params), int(momentum), float(lr), float(beta), int(prev_agg),
+                                  int(partials) if partials else None, int(stream) if stream else None)
+
+
+def dmx_step_adam_partial(h, grad_ptrs, batch_sizes, params, first_moment, second_moment, lr, beta1, beta2, eps, t,
+                          prev_agg, partials, stream=0) -> int:
+    K = len(grad_ptrs)
+    gp = (ctypes.c_void_p * K)(*[int(p) for p in grad_ptrs])
+    bs = (ctypes.c_int32 * K)(*[int(b) for b in batch_sizes])
+    return lib().dmx_step_adam_partial(h, gp, bs, int(params), int(first_moment), int(second_moment), float(lr),
+                                       float(beta1), float(beta2), float(eps), int(t), int(prev_agg),
+                                       int(partials) if partials else None, int(stream) if stream else None)
+
+
+def dmx_finalize_partials(K, S, batch_sizes, partials, adam, P_total, out_state, stream=0) -> int:
+    """The state vector from the shards' summed partials (device addresses)."""
+    bs = (ctypes.c_int32 * len(batch_sizes))(*[int(b) for b in batch_sizes])
+    return lib().dmx_finalize_partials(int(K), int(S), bs, int(partials) if partials else None, int(bool(adam)),
+                                       int(P_total), int(out_state) if out_state else None,
+                                       int(stream) if stream else None)
+
+
 def dmx_plan_chunks(P, K, grad_dtype, tile_elems, resident_ctas):
     """-> (code_or_count, first_tile, num_tiles, group_stride, group_tiles, grid): the fused pass's work
     list as dmx_create would build it (host only; lists of ints)."""
@@ -337,6 +398,76 @@ class Dmx:
     @property
     def launches_per_step(self):
         return dmx_launches_per_step(self._h)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            dmx_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+
+class ShardedDmx:
+    """One parameter shard of a problem (shard `shard` of `nshards`), for torch callers.
+
+    `step_partial` runs the fused pass on views [lo:hi) of the full-length tensors and returns the
+    shard's raw sums (a float64 device tensor); the caller adds the shards' tensors (an all-reduce
+    when the shards live on different GPUs, see dist_util.allreduce_sum) and calls `finalize`.
+    """
+
+    def __init__(self, K, P, seg_offsets, grad_dtype, nshards, shard):
+        import torch
+        self._torch = torch
+        self.K, self.P, self.S, self.dtype = int(K), int(P), len(seg_offsets) - 1, int(grad_dtype)
+        rc, self.lo, self.hi = dmx_shard_range(P, nshards, shard)
+        if rc != OK:
+            raise DmxError(rc, "dmx_shard_range")
+        self.state_len = ST_HDR + self.K + 2 * self.S
+        self.partials_len = self.K + 5 + 2 * self.S
+        self._h = None
+        if self.hi > self.lo:
+            rc, seg = dmx_shard_segments(seg_offsets, self.lo, self.hi)
+            if rc != OK:
+                raise DmxError(rc, "dmx_shard_segments")
+            rc, self._h = dmx_create(K, self.hi - self.lo, seg, grad_dtype)
+            if rc != OK:
+                self._h = None
+                raise DmxError(rc, "dmx_create")
+
+    def step_partial(self, grads, batch_sizes, params, momentum, lr, beta, prev_agg, adam=None, stream=None):
+        """adam: None for SGD with momentum, else (second_moment, beta2, eps, t) with beta = beta1."""
+        torch = self._torch
+        part = torch.zeros(self.partials_len, dtype=torch.float64, device=params.device)
+        if self._h is None:                      # an empty shard contributes zeros
+            return part
+        if stream is None:
+            stream = torch.cuda.current_stream(params.device).cuda_stream
+        esz = 2 if self.dtype == BF16 else 4
+        gp = [g.data_ptr() + self.lo * esz for g in grads]
+        off = self.lo * 4
+        if adam is None:
+            rc = dmx_step_partial(self._h, gp, batch_sizes, params.data_ptr() + off, momentum.data_ptr() + off, lr, beta,
+                                  prev_agg.data_ptr() + off, part.data_ptr(), stream)
+        else:
+            second, beta2, eps, t = adam
+            rc = dmx_step_adam_partial(self._h, gp, batch_sizes, params.data_ptr() + off, momentum.data_ptr() + off,
+                                       second.data_ptr() + off, lr, beta, beta2, eps, t, prev_agg.data_ptr() + off,
+                                       part.data_ptr(), stream)
+        if rc != OK:
+            raise DmxError(rc, "dmx_step_partial")
+        return part
+
+    def finalize(self, batch_sizes, partials_sum, adam=False, out_state=None, stream=None):
+        torch = self._torch
+        if out_state is None:
+            out_state = torch.empty(self.state_len, dtype=torch.float32, device=partials_sum.device)
+        if stream is None:
+            stream = torch.cuda.current_stream(partials_sum.device).cuda_stream
+        rc = dmx_finalize_partials(self.K, self.S, batch_sizes, partials_sum.data_ptr(), adam, self.P,
+                                   out_state.data_ptr(), stream)
+        if rc != OK:
+            raise DmxError(rc, "dmx_finalize_partials")
+        return out_state
 
     def close(self):
         if getattr(self, "_h", None):

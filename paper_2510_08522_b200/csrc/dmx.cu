@@ -166,7 +166,8 @@ struct ChunkPlan {
   std::vector<int32_t> tile0, ntiles, stride;   // per chunk: first tile, tiles, tiles between group starts
 };
 
-void plan_chunks(int64_t P, int K, int grad_dtype, int tile, int64_t sm_ctas, int want_R, int want_chunk, ChunkPlan& cp) {
+void plan_chunks(int64_t P, int K, int grad_dtype, int tile, int64_t sm_ctas, int want_R, int want_chunk, int want_min_kb,
+                 ChunkPlan& cp) {
   const int64_t ntiles = (P + tile - 1) / tile;
   const int auto_R = ntiles >= 4 * 64 * sm_ctas ? 4 : (ntiles >= 32 * sm_ctas ? 2 : 1);
   const int R = std::max(1, std::min(want_R > 0 ? want_R : auto_R, 1 << 16));          // tiles per group
@@ -182,7 +183,8 @@ void plan_chunks(int64_t P, int K, int grad_dtype, int tile, int64_t sm_ctas, in
   // smallest chunk: about 192 KB of streamed bytes (a few microseconds of one SM), so that the
   // per-chunk work (the draw, the reduction flush) stays small beside it
   const int64_t group_bytes = (int64_t)R * tile * ((int64_t)K * (grad_dtype == DMX_BF16 ? 2 : 4) + 24);
-  const int64_t min_groups = std::min<int64_t>(chunk_groups, std::max<int64_t>(1, (192 * 1024 + group_bytes - 1) / group_bytes));
+  const int64_t min_bytes = (int64_t)(want_min_kb > 0 ? want_min_kb : 192) * 1024;
+  const int64_t min_groups = std::min<int64_t>(chunk_groups, std::max<int64_t>(1, (min_bytes + group_bytes - 1) / group_bytes));
   for (int64_t g0 = 0; g0 < ngroups;) {
     const int64_t rem = ngroups - g0;
     // a problem of less than two minimum chunks per CTA is one wave, split evenly (nothing to balance)
@@ -274,7 +276,8 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   const int64_t ntiles = (P + plan.tile - 1) / plan.tile;
   const int64_t sm_ctas = (int64_t)prop.multiProcessorCount * occ;
   ChunkPlan cp;
-  plan_chunks(P, K, grad_dtype, plan.tile, sm_ctas, env_int("DMX_TILE_GROUP", 0), env_int("DMX_CHUNK_TILES", 0), cp);
+  plan_chunks(P, K, grad_dtype, plan.tile, sm_ctas, env_int("DMX_TILE_GROUP", 0), env_int("DMX_CHUNK_TILES", 0),
+              env_int("DMX_MIN_CHUNK_KB", 0), cp);
   const int R = cp.R;
   plan.grid = cp.grid;
   h->plan = plan;
@@ -370,16 +373,18 @@ struct AdamParams { float* second; float beta2, eps; int64_t t; };
 // One step with either update; `ap` is null for SGD with momentum.
 int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes, float* params,
               float* momentum, float lr, float beta, float* prev_agg, float* out_state, void* cuda_stream,
-              const AdamParams* ap) {
+              const AdamParams* ap, double* partials = nullptr) {
+  // `partials` (a parameter shard of a larger problem): the raw sums go there and out_state is not written
   if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
-  if (!grad_ptrs || !batch_sizes || !params || !momentum || !prev_agg || !out_state) return DMX_ERR_ARG;
+  if (!grad_ptrs || !batch_sizes || !params || !momentum || !prev_agg || (!out_state && !partials)) return DMX_ERR_ARG;
   if (ap && (!ap->second || ap->t < 1 || !(beta >= 0.f && beta < 1.f) || !(ap->beta2 >= 0.f && ap->beta2 < 1.f) ||
              !(ap->eps >= 0.f)))
     return DMX_ERR_ARG;
   const int K = h->K;
   const size_t esz = h->dtype == DMX_BF16 ? 2 : 4;
   const size_t gbytes = (size_t)h->P * esz, sbytes = (size_t)h->P * 4;
-  const size_t obytes = (size_t)(DMX_ST_HDR + K + 2 * h->S) * 4;
+  const size_t obytes = partials ? (size_t)(K + 5 + 2 * h->S) * 8 : (size_t)(DMX_ST_HDR + K + 2 * h->S) * 4;
+  const void* outp = partials ? (const void*)partials : (const void*)out_state;
   int64_t B = 0;
   int pivot = 0;
   for (int k = 0; k < K; ++k) {
@@ -390,10 +395,11 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
   }
   for (int k = 0; k < K; ++k)
     if ((uintptr_t)grad_ptrs[k] & 15) return DMX_ERR_ALIGN;
-  if (((uintptr_t)params & 15) || ((uintptr_t)momentum & 15) || ((uintptr_t)prev_agg & 15) || ((uintptr_t)out_state & 3))
+  if (((uintptr_t)params & 15) || ((uintptr_t)momentum & 15) || ((uintptr_t)prev_agg & 15) ||
+      ((uintptr_t)outp & (partials ? 7 : 3)))
     return DMX_ERR_ALIGN;
   if (ap && ((uintptr_t)ap->second & 15)) return DMX_ERR_ALIGN;
-  const void* st[5] = {params, momentum, prev_agg, out_state, ap ? ap->second : nullptr};
+  const void* st[5] = {params, momentum, prev_agg, outp, ap ? ap->second : nullptr};
   const size_t sn[5] = {sbytes, sbytes, sbytes, obytes, sbytes};
   const int nst = ap ? 5 : 4;
   for (int i = 0; i < nst; ++i) {
@@ -442,6 +448,7 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
   F.rows = h->rows; F.slots = h->slots; F.seg_slots = h->seg_slots; F.nunits = h->nunits;
   F.unit_lo = h->unit_lo; F.unit_hi = h->unit_hi; F.seg_unit_ptr = h->seg_unit_ptr; F.segpart = h->segpart;
   F.colsum = h->colsum; F.ticket = h->flags; F.err = h->flags + 1; F.out_state = out_state;
+  F.partials = partials;
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const bool prof = h->profiling;
@@ -489,6 +496,68 @@ int dmx_step_adam(dmx_handle* h, const void* const* grad_ptrs, const int32_t* ba
                   int64_t t, float* prev_agg, float* out_state, void* cuda_stream) {
   const AdamParams ap = {second_moment, beta2, eps, t};
   return step_impl(h, grad_ptrs, batch_sizes, params, first_moment, lr, beta1, prev_agg, out_state, cuda_stream, &ap);
+}
+
+int dmx_partials_len(const dmx_handle* h) {
+  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
+  return h->K + 5 + 2 * h->S;
+}
+
+int dmx_step_partial(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes, float* params,
+                     float* momentum, float lr, float beta, float* prev_agg, double* partials, void* cuda_stream) {
+  if (!partials) return DMX_ERR_ARG;
+  return step_impl(h, grad_ptrs, batch_sizes, params, momentum, lr, beta, prev_agg, nullptr, cuda_stream, nullptr, partials);
+}
+
+int dmx_step_adam_partial(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes, float* params,
+                          float* first_moment, float* second_moment, float lr, float beta1, float beta2, float eps,
+                          int64_t t, float* prev_agg, double* partials, void* cuda_stream) {
+  if (!partials) return DMX_ERR_ARG;
+  const AdamParams ap = {second_moment, beta2, eps, t};
+  return step_impl(h, grad_ptrs, batch_sizes, params, first_moment, lr, beta1, prev_agg, nullptr, cuda_stream, &ap, partials);
+}
+
+int dmx_finalize_partials(int K, int S, const int32_t* batch_sizes, const double* partials, int adam, int64_t P_total,
+                          float* out_state, void* cuda_stream) {
+  if (K < 1 || K > DMX_MAX_WORKERS || S < 1 || S > DMX_MAX_SEGMENTS || !batch_sizes || !partials || !out_state ||
+      P_total < 1 || P_total >= DMX_MAX_PARAMS)
+    return DMX_ERR_ARG;
+  if (((uintptr_t)partials & 7) || ((uintptr_t)out_state & 3)) return DMX_ERR_ALIGN;
+  dmx::DeriveArgs G;
+  std::memset(&G, 0, sizeof(G));
+  int64_t B = 0;
+  for (int k = 0; k < K; ++k) {
+    if (batch_sizes[k] < 1) return DMX_ERR_BATCH;
+    G.b[k] = (double)batch_sizes[k];
+    B += batch_sizes[k];
+  }
+  G.K = K; G.S = S; G.adam = adam ? 1 : 0; G.P = (double)P_total; G.B = (double)B;
+  G.partials = partials; G.out_state = out_state;
+  dmx::derive_kernel<<<1, dmx::kFinalWarps * 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(G);
+  if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
+  return DMX_OK;
+}
+
+int dmx_shard_range(int64_t P, int nshards, int shard, int64_t* lo, int64_t* hi) {
+  if (P < 1 || nshards < 1 || shard < 0 || shard >= nshards || !lo || !hi) return DMX_ERR_ARG;
+  // boundaries on multiples of 1024 elements: shard pointers keep their 16-byte alignment for either
+  // gradient type; a shard may be empty when P is small
+  const int64_t align = 1024;
+  const int64_t units = (P + align - 1) / align;
+  const int64_t a = units * shard / nshards * align, b = units * (shard + 1) / nshards * align;
+  *lo = std::min<int64_t>(a, P);
+  *hi = shard == nshards - 1 ? P : std::min<int64_t>(b, P);
+  return DMX_OK;
+}
+
+int dmx_shard_segments(const int64_t* seg_offsets, int S, int64_t lo, int64_t hi, int64_t* shard_offsets) {
+  if (!seg_offsets || !shard_offsets || S < 1 || S > DMX_MAX_SEGMENTS || lo < 0 || hi < lo) return DMX_ERR_ARG;
+  if (seg_offsets[0] != 0 || hi > seg_offsets[S]) return DMX_ERR_SEGMENTS;
+  for (int s = 0; s <= S; ++s) {
+    if (s < S && seg_offsets[s] > seg_offsets[s + 1]) return DMX_ERR_SEGMENTS;
+    shard_offsets[s] = std::min<int64_t>(std::max<int64_t>(seg_offsets[s], lo), hi) - lo;
+  }
+  return DMX_OK;
 }
 
 int dmx_step_host(dmx_handle* h, const void* const* host_grad_ptrs, void* const* staging_ptrs,
@@ -540,7 +609,7 @@ int dmx_plan_chunks(int64_t P, int K, int grad_dtype, int tile_elems, int reside
       (grad_dtype != DMX_F32 && grad_dtype != DMX_BF16) || capacity < 0)
     return DMX_ERR_ARG;
   ChunkPlan cp;
-  plan_chunks(P, K, grad_dtype, tile_elems, resident_ctas, 0, 0, cp);
+  plan_chunks(P, K, grad_dtype, tile_elems, resident_ctas, 0, 0, 0, cp);
   if (group_tiles) *group_tiles = cp.R;
   if (grid) *grid = cp.grid;
   const int n = (int)cp.tile0.size();

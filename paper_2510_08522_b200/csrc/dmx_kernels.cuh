@@ -86,6 +86,19 @@ struct FinalArgs {
   unsigned* ticket;
   unsigned* err;
   float* out_state;
+  double* partials;            // not null: emit the raw fp64 sums of this parameter shard instead of out_state
+};
+
+// Raw sums of a step over a parameter range, as dmx_step_partial emits them (K + 5 + 2 S doubles):
+// q_k in the caller's worker order [K], <g,a>, |a|^2, Adam's sum and sum of squares of ghat (0
+// otherwise), Vraw_s [S], N_s [S], and a word that is non-zero if a bounded wait ran out.
+// Shards of one problem add up entry by entry.
+struct DeriveArgs {
+  int K, S, adam;
+  double P, B;
+  double b[kMaxK];             // batch sizes, caller's order
+  const double* partials;
+  float* out_state;
 };
 
 typedef unsigned long long u64;
@@ -506,6 +519,35 @@ __device__ __forceinline__ double warp_sum_d(double v) {
 
 constexpr int kFinalWarps = 8;
 
+// The scalar part of the state vector from the step's reduced sums (the definitions of the state
+// layout): D = sum_s Vraw_s, A = sum_s N_s, Qw = sum_k b_k q_k, c = <g,a>, pp = |a|^2.
+__device__ __forceinline__ void emit_header(float* out, int K, double B, double D, double A, double Qw, double c, double pp,
+                                            bool nonfinite_q, bool internal, int adam, double su, double su2, double P) {
+  int flags = 0;
+  double trS = 0.0;
+  if (K >= 2) trS = D / (double)(K - 1); else flags |= 8;
+  const double G2 = A - trS / B;
+  double gns = 0.0;
+  if (G2 > 0.0) gns = trS / G2; else flags |= 2;
+  double cosv = 0.0;
+  if (A > 0.0 && pp > 0.0) cosv = c / sqrt(A * pp); else flags |= 4;
+  const double sig2 = A > 0.0 ? trS / (B * A) : 0.0;
+  const double sig = sqrt(sig2 > 0.0 ? sig2 : 0.0);
+  if (nonfinite_q || !isfinite((float)A) || !isfinite((float)pp)) flags |= 1;
+  if (internal) flags |= 16;
+  out[0] = (float)B; out[1] = (float)A; out[2] = (float)trS; out[3] = (float)G2; out[4] = (float)gns;
+  out[5] = (float)cosv; out[6] = (float)c; out[7] = (float)pp; out[8] = (float)sig2; out[9] = (float)sig;
+  out[10] = (float)(Qw / B); out[11] = (float)flags;
+  out[12] = out[13] = out[14] = out[15] = 0.f;
+  if (adam) {
+    // the gradient in units of Adam's running scale, ghat_j = g_j / (sqrt(vhat_j) + eps):
+    // its mean, variance and standard deviation across the parameters
+    const double mean = su / P;
+    const double var = su2 / P - mean * mean;
+    out[12] = (float)mean; out[13] = (float)var; out[14] = (float)sqrt(var > 0.0 ? var : 0.0);
+  }
+}
+
 constexpr int kFinalPart = 256;  // slots per segment unit
 
 // First level. Blocks 0..ncol-1 each sum one column (q_k, c, pp, and Adam's two) of the chunk
@@ -578,6 +620,27 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
     if (threadIdx.x < ncol) cs[threadIdx.x] = gcs[threadIdx.x];
   }
   const volatile double2* sp = F.segpart;
+  if (F.partials) {
+    // a parameter shard of a larger problem: hand out the raw sums, to be added over the shards
+    double* pt = F.partials;
+    for (int s = threadIdx.x; s < S; s += blockDim.x) {
+      double v = 0.0, n = 0.0;
+      for (int u = F.seg_unit_ptr[s]; u < F.seg_unit_ptr[s + 1]; ++u) { v += sp[u].x; n += sp[u].y; }
+      pt[K + 4 + s] = v;
+      pt[K + 4 + S + s] = n;
+    }
+    __syncthreads();                                   // cs[] is in place
+    for (int k = threadIdx.x; k < K; k += blockDim.x) pt[F.orig[k]] = cs[k];
+    if (threadIdx.x == 0) {
+      pt[K] = cs[K]; pt[K + 1] = cs[K + 1];
+      pt[K + 2] = F.adam ? cs[K + 2] : 0.0; pt[K + 3] = F.adam ? cs[K + 3] : 0.0;
+      const bool internal = *reinterpret_cast<volatile unsigned*>(F.err) != 0u;
+      pt[K + 4 + 2 * S] = internal ? 1.0 : 0.0;
+      if (internal) *F.err = 0u;
+      *F.ticket = 0u;
+    }
+    return;
+  }
   float* out = F.out_state;
   double aV = 0.0, aN = 0.0;
   for (int s = threadIdx.x; s < S; s += blockDim.x) {
@@ -596,31 +659,38 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
     for (int w = 0; w < kFinalWarps; ++w) { D += s_red[0][w]; A += s_red[1][w]; }
     bool bad = false;
     for (int k = 0; k < K; ++k) { const double qk = cs[k]; Qw += F.b[k] * qk; bad = bad | !isfinite((float)qk); }
-    const double c = cs[K], pp = cs[K + 1], B = F.B;
-    int flags = 0;
-    double trS = 0.0;
-    if (K >= 2) trS = D / (double)(K - 1); else flags |= 8;
-    const double G2 = A - trS / B;
-    double gns = 0.0;
-    if (G2 > 0.0) gns = trS / G2; else flags |= 2;
-    double cosv = 0.0;
-    if (A > 0.0 && pp > 0.0) cosv = c / sqrt(A * pp); else flags |= 4;
-    const double sig2 = A > 0.0 ? trS / (B * A) : 0.0;
-    const double sig = sqrt(sig2 > 0.0 ? sig2 : 0.0);
-    if (bad || !isfinite((float)A) || !isfinite((float)pp)) flags |= 1;
-    if (*reinterpret_cast<volatile unsigned*>(F.err) != 0u) { flags |= 16; *F.err = 0u; }
-    out[0] = (float)B; out[1] = (float)A; out[2] = (float)trS; out[3] = (float)G2; out[4] = (float)gns;
-    out[5] = (float)cosv; out[6] = (float)c; out[7] = (float)pp; out[8] = (float)sig2; out[9] = (float)sig;
-    out[10] = (float)(Qw / B); out[11] = (float)flags;
-    out[12] = out[13] = out[14] = out[15] = 0.f;
-    if (F.adam) {
-      // the gradient in units of Adam's running scale, ghat_j = g_j / (sqrt(vhat_j) + eps):
-      // its mean, variance and standard deviation across the parameters
-      const double mean = cs[K + 2] / F.P;
-      const double var = cs[K + 3] / F.P - mean * mean;
-      out[12] = (float)mean; out[13] = (float)var; out[14] = (float)sqrt(var > 0.0 ? var : 0.0);
-    }
+    const bool internal = *reinterpret_cast<volatile unsigned*>(F.err) != 0u;
+    if (internal) *F.err = 0u;
+    emit_header(out, K, F.B, D, A, Qw, cs[K], cs[K + 1], bad, internal, F.adam, F.adam ? cs[K + 2] : 0.0,
+                F.adam ? cs[K + 3] : 0.0, F.P);
     *F.ticket = 0u;
+  }
+}
+
+// The state vector from raw sums added over the parameter shards of one problem (one block).
+static __global__ void __launch_bounds__(kFinalWarps * 32) derive_kernel(const __grid_constant__ DeriveArgs G) {
+  const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int K = G.K, S = G.S;
+  const double* pt = G.partials;
+  float* out = G.out_state;
+  __shared__ double s_red[2][kFinalWarps];
+  double aV = 0.0, aN = 0.0;
+  for (int s = threadIdx.x; s < S; s += blockDim.x) {
+    const double v = pt[K + 4 + s], n = pt[K + 4 + S + s];
+    out[16 + K + s] = K >= 2 ? (float)(v / (double)(K - 1)) : 0.f;
+    out[16 + K + S + s] = (float)n;
+    aV += v; aN += n;
+  }
+  aV = warp_sum_d(aV); aN = warp_sum_d(aN);
+  if (lane == 0) { s_red[0][wid] = aV; s_red[1][wid] = aN; }
+  __syncthreads();
+  for (int k = threadIdx.x; k < K; k += blockDim.x) out[16 + k] = (float)pt[k];
+  if (threadIdx.x == 0) {
+    double D = 0.0, A = 0.0, Qw = 0.0;
+    for (int w = 0; w < kFinalWarps; ++w) { D += s_red[0][w]; A += s_red[1][w]; }
+    bool bad = false;
+    for (int k = 0; k < K; ++k) { const double qk = pt[k]; Qw += G.b[k] * qk; bad = bad | !isfinite((float)qk); }
+    emit_header(out, K, G.B, D, A, Qw, pt[K], pt[K + 1], bad, pt[K + 4 + 2 * S] != 0.0, G.adam, pt[K + 2], pt[K + 3], G.P);
   }
 }
 

@@ -1,7 +1,9 @@
-"""Process-group plumbing for running N independent replicas of the step (one process per GPU).
+"""Process-group plumbing for running the step on N GPUs (one process per GPU).
 
-The gradient step has no exchange between GPUs: K workers are emulated on each GPU, so N GPUs
-run N replicas and the only collectives are the barrier and the max-over-ranks of the timings.
+Replicas: the gradient step has no exchange between GPUs when each GPU emulates its own K
+workers, so N GPUs run N replicas and the only collectives are the barrier and the
+max-over-ranks of the timings. Parameter shards of ONE problem (ShardedDmx) have one exchange
+step: the sum of the shards' raw fp64 sums (`allreduce_sum`).
 """
 from __future__ import annotations
 
@@ -38,6 +40,15 @@ def max_over_ranks(x: float) -> float:
     t = torch.tensor([float(x)], dtype=torch.float64, device=dev)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def allreduce_sum(t):
+    """Entry-wise sum over the ranks of a tensor (the shards' partial sums), in place; the
+    tensor lives where the backend wants it (device memory for nccl, host memory for gloo)."""
+    if _world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return t
 
 
 def job_throughput(units_per_rank: float, local_ms: float) -> float:
