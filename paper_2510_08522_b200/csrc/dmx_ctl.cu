@@ -17,6 +17,8 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kMaxF = DMX_CTL_MAX_AUX + DMX_CTL_LOCAL_EXTRA + DMX_CTL_GLOBAL_FEATURES;
+constexpr int kMaxIn = DMX_CTL_MAX_HIDDEN;     // longest input vector of a layer
+static_assert(kMaxF <= kMaxIn && kMaxIn % 32 == 0, "a layer's input fits the per-lane weight registers");
 
 struct CtlArgs {
   int K, M, H, state_len;
@@ -35,10 +37,47 @@ struct CtlArgs {
   float* features;  // K x F, or null
 };
 
+// One layer, a warp per group of four output rows (four independent chains of loads in flight:
+// the layer is latency-bound): out[r] = sum_j W[r][j] x[j] + c[r] for r < rows, fp64, lanes
+// striding through the row (coalesced weight loads), then a shuffle tree in a fixed order. The
+// activation is applied afterwards by one thread per row (fp64 tanh is a long dependent chain:
+// 32 of them in a row on one lane cost more than the dot products).
+__device__ __forceinline__ void layer(const float* __restrict__ W, const float* __restrict__ c, const double* x,
+                                      double* out, int rows, int n, int wid, int lane) {
+  for (int r0 = wid * 4; r0 < rows; r0 += (kThreads / 32) * 4) {
+    double s[4] = {0.0, 0.0, 0.0, 0.0};
+    // all of the group's weights are requested before the first one is used (n <= 256: at most
+    // eight per lane and row)
+    float w[4][kMaxIn / 32];
+#pragma unroll
+    for (int it = 0; it < kMaxIn / 32; ++it) {
+      const int j = lane + 32 * it;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) w[q][it] = (j < n && r0 + q < rows) ? W[(size_t)(r0 + q) * n + j] : 0.f;
+    }
+#pragma unroll
+    for (int it = 0; it < kMaxIn / 32; ++it) {
+      const int j = lane + 32 * it;
+      const double xj = j < n ? x[j] : 0.0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) s[q] = fma((double)w[q][it], xj, s[q]);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) s[q] += __shfl_xor_sync(0xffffffffu, s[q], o);
+      if (lane == 0 && r0 + q < rows) {
+        out[r0 + q] = s[q] + (double)c[r0 + q];
+      }
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kThreads) ctl_kernel(const CtlArgs A) {
   __shared__ double f[kMaxF];
   __shared__ double h1[DMX_CTL_MAX_HIDDEN], h2[DMX_CTL_MAX_HIDDEN];
   __shared__ float z[DMX_CTL_ACTIONS];
+  __shared__ double zd[8];
   const int i = blockIdx.x, t = threadIdx.x;
   const int M = A.M, H = A.H, F = M + DMX_CTL_LOCAL_EXTRA + DMX_CTL_GLOBAL_FEATURES;
   const float* mean = A.window;
@@ -78,23 +117,20 @@ __global__ void __launch_bounds__(kThreads) ctl_kernel(const CtlArgs A) {
   const float* c2 = W2 + (size_t)H * H;
   const float* W3 = c2 + H;
   const float* c3 = W3 + (size_t)DMX_CTL_ACTIONS * H;
-  if (t < H) {
-    double s = (double)c1[t];
-    for (int j = 0; j < F; ++j) s = fma((double)W1[(size_t)t * F + j], f[j], s);
-    h1[t] = tanh(s);
-  }
+  const int wid = t >> 5, lane = t & 31;
+  layer(W1, c1, f, h1, H, F, wid, lane);
   __syncthreads();
-  if (t < H) {
-    double s = (double)c2[t];
-    for (int j = 0; j < H; ++j) s = fma((double)W2[(size_t)t * H + j], h1[j], s);
-    h2[t] = tanh(s);
-  }
+  if (t < H) h1[t] = tanh(h1[t]);
+  __syncthreads();
+  layer(W2, c2, h1, h2, H, H, wid, lane);
+  __syncthreads();
+  if (t < H) h2[t] = tanh(h2[t]);
+  __syncthreads();
+  layer(W3, c3, h2, zd, DMX_CTL_ACTIONS, H, wid, lane);
   __syncthreads();
   if (t < DMX_CTL_ACTIONS) {
-    double s = (double)c3[t];
-    for (int j = 0; j < H; ++j) s = fma((double)W3[(size_t)t * H + j], h2[j], s);
-    z[t] = (float)s;
-    A.logits[(size_t)i * DMX_CTL_ACTIONS + t] = (float)s;
+    z[t] = (float)zd[t];
+    A.logits[(size_t)i * DMX_CTL_ACTIONS + t] = (float)zd[t];
   }
   __syncthreads();
   if (t != 0) return;
