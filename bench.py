@@ -114,6 +114,10 @@ class ClockSampler:
         return out
 
 
+def world_is_one():
+    return int(os.environ.get("WORLD_SIZE", "1")) == 1
+
+
 def step_bytes(wl, optimizer):
     """Algorithmic HBM bytes of one step (Adam reads and writes one more fp32 state stream)."""
     return wl.bytes_per_step + (8 * wl.P if optimizer == "adam" else 0)
@@ -207,6 +211,12 @@ def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profi
         res["e2e_launches"] = e2e_steps * d.launches_per_step
         del host
     d.close()
+    if sample_clocks and world_is_one():
+        # what plain reads of the same gradient buffers stream at in this run (context for the roofline)
+        try:
+            res["read_probe_gbps"] = W.read_probe_gbps(dp.grads)
+        except Exception:
+            res["read_probe_gbps"] = None
     res["problem"] = dp
     return res
 
@@ -369,6 +379,9 @@ def main():
                          "traffic": recorded_traffic(wl.name) if args.optimizer == "sgd" else None,
                          "algorithmic_bytes_per_launch": nbytes},
             "internal_error_flag": bool(flags_any)}
+    if res.get("read_probe_gbps"):
+        line["roofline"]["read_only_probe"] = {"value": res["read_probe_gbps"], "unit": UNIT,
+                                               "what": "plain 128-bit reads of the same K gradient buffers, same run"}
     if "e2e_ms" in res:
         line["e2e"] = {"value": world * wl.bytes_per_step / e2e_ms / 1e6, "unit": UNIT,
                        "h2d_bytes_per_step": res["h2d_bytes"], "d2h_bytes_per_step": res["d2h_bytes"],

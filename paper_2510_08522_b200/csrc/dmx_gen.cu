@@ -89,9 +89,44 @@ int launch(void* dst, const float* base, float mean, float scale, int64_t n, int
   return cudaGetLastError() == cudaSuccess ? 0 : -6;
 }
 
+// Read-only streaming probe: every thread reads 16-byte pieces of up to 64 buffers with eight
+// loads in flight and folds them into a checksum (one word per CTA). It measures what the
+// memory system delivers for plain reads of the benchmark's own buffers.
+struct ProbeArgs { const uint4* src[64]; int nsrc; long long n16; uint32_t* sink; };
+
+__global__ void __launch_bounds__(256) read_probe_kernel(const __grid_constant__ ProbeArgs A) {
+  uint32_t acc = 0;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < A.n16; i += stride) {
+#pragma unroll 8
+    for (int k = 0; k < A.nsrc; ++k) {
+      uint4 v;
+      asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(A.src[k] + i));
+      acc ^= v.x + v.y + v.z + v.w;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc ^= __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0) atomicXor(A.sink + blockIdx.x, acc);
+}
+
 }  // namespace
 
 extern "C" {
+
+// Reads `bytes` bytes (a multiple of 16) of each of nsrc DEVICE buffers (16-byte aligned) once;
+// sink: DEVICE, at least 148 * 8 words, receives checksums. Returns 0 or a negative code.
+int dmxgen_read_probe(const void* const* src, int nsrc, int64_t bytes, uint32_t* sink, void* stream) {
+  if (!src || nsrc < 1 || nsrc > 64 || bytes < 16 || (bytes & 15) || !sink) return -1;
+  ProbeArgs A;
+  for (int k = 0; k < nsrc; ++k) {
+    if (!src[k] || (reinterpret_cast<uintptr_t>(src[k]) & 15)) return -4;
+    A.src[k] = static_cast<const uint4*>(src[k]);
+  }
+  A.nsrc = nsrc; A.n16 = bytes / 16; A.sink = sink;
+  read_probe_kernel<<<148 * 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(A);
+  return cudaGetLastError() == cudaSuccess ? 0 : -6;
+}
 
 // dst[j] = mean + std * z_j                                  (fp32, DEVICE, 16-byte aligned)
 int dmxgen_normal_fill(float* dst, int64_t n, uint32_t seed, uint32_t tag, uint32_t c2, uint32_t c3,

@@ -273,7 +273,8 @@ def gen_lib():
         L.dmxgen_normal_fill.argtypes = [vp, i64, u32, u32, u32, u32, f32, f32, vp]
         L.dmxgen_normal_add.argtypes = [vp, i64, u32, u32, u32, u32, f32, vp]
         L.dmxgen_grad_fill.argtypes = [vp, i32, vp, i64, u32, u32, u32, u32, f32, vp]
-        for f in (L.dmxgen_normal_fill, L.dmxgen_normal_add, L.dmxgen_grad_fill):
+        L.dmxgen_read_probe.argtypes = [vp, i32, i64, vp, vp]
+        for f in (L.dmxgen_normal_fill, L.dmxgen_normal_add, L.dmxgen_grad_fill, L.dmxgen_read_probe):
             f.restype = i32
         _gen = L
     return _gen
@@ -335,3 +336,29 @@ class DeviceProblem:
             with self.torch.cuda.device(self.device):
                 self._chk(gen_lib().dmxgen_normal_add(self.mu.data_ptr(), self.wl.P, self.wl.seed, TAG_DRIFT, 0,
                                                       self.step_index, DRIFT_STD, self._stream()), "drift")
+
+
+def read_probe_gbps(tensors, reps=5):
+    """Read-only streaming rate (GB/s) over the given equally sized device tensors: the median of
+    `reps` timed passes of the generator library's probe kernel after one warm-up pass."""
+    import ctypes
+    import torch
+    L = gen_lib()
+    n = len(tensors)
+    nbytes = min(t.numel() * t.element_size() for t in tensors) // 16 * 16
+    ptrs = (ctypes.c_void_p * n)(*[t.data_ptr() for t in tensors])
+    sink = torch.zeros(148 * 8, dtype=torch.int32, device=tensors[0].device)
+    stream = torch.cuda.current_stream(tensors[0].device).cuda_stream
+    ts = []
+    for i in range(reps + 1):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        rc = L.dmxgen_read_probe(ptrs, n, nbytes, sink.data_ptr(), stream)
+        e1.record()
+        torch.cuda.synchronize()
+        if rc != 0:
+            raise RuntimeError("dmxgen_read_probe failed: %d" % rc)
+        if i:
+            ts.append(e0.elapsed_time(e1))
+    ts.sort()
+    return n * nbytes / ts[len(ts) // 2] / 1e6

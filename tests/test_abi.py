@@ -27,7 +27,7 @@ def test_library_is_built_and_exports_every_declared_symbol():
     for n in names:
         assert hasattr(lib, n), n
     gen = ctypes.CDLL(build.lib_path("libdmx_gen.so"))
-    for n in ("dmxgen_normal_fill", "dmxgen_normal_add", "dmxgen_grad_fill"):
+    for n in ("dmxgen_normal_fill", "dmxgen_normal_add", "dmxgen_grad_fill", "dmxgen_read_probe"):
         assert hasattr(gen, n)
 
 
