@@ -22,6 +22,9 @@
  *     not allocate, does not synchronise and copies nothing host-to-device (worker pointers,
  *     weights and batch sizes travel as kernel arguments).
  *   - A handle may be used from one stream at a time (its scratch is shared by its calls).
+ *   - dmx_step, dmx_step_adam and their _partial forms enqueue two kernel launches and nothing
+ *     else, so (with per-kernel timing off) they can be captured in a CUDA graph and replayed:
+ *     the kernels leave the handle's scratch ready for the next run.
  */
 #ifndef DMX_H_
 #define DMX_H_

@@ -67,8 +67,7 @@ struct dmx_handle {
   float* rows = nullptr;
   float2* slots = nullptr;
   double* colsum = nullptr;
-  unsigned* flags = nullptr;  // [0] ticket, [1] err, [2] and [3] chunk counters of even and odd steps
-  unsigned step_parity = 0;   // which chunk counter the next step draws from
+  unsigned* flags = nullptr;  // [0] ticket, [1] err, [2] the fused pass's chunk counter
   // optional per-kernel timing
   bool profiling = false, profiled = false;
   cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
@@ -437,8 +436,9 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
   }
   A.K = K; A.S = h->S; A.P = h->P;
   A.tile_group = h->tile_group; A.nchunks = h->nchunks;
-  // the step's chunk counter is zero: the previous step's kernel reset it while it drew from the other one
-  A.next_chunk = h->flags + 2 + h->step_parity; A.next_chunk_reset = h->flags + 2 + (h->step_parity ^ 1u);
+  // the chunk counter is zero here: the finalize kernel of the previous step (or dmx_create) left it so,
+  // which also makes a step that was captured in a CUDA graph replayable
+  A.next_chunk = h->flags + 2;
   A.seg_off = h->seg_off; A.tile_seg = h->tile_seg; A.chunk_stride = h->chunk_stride; A.chunk_tile0 = h->chunk_tile0;
   A.chunk_ntiles = h->chunk_ntiles; A.chunk_slot0 = h->chunk_slot0;
   A.rows = h->rows; A.slots = h->slots; A.err = h->flags + 1;
@@ -447,7 +447,8 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
   F.adam = ap ? 1 : 0; F.P = (double)h->P;
   F.rows = h->rows; F.slots = h->slots; F.seg_slots = h->seg_slots; F.nunits = h->nunits;
   F.unit_lo = h->unit_lo; F.unit_hi = h->unit_hi; F.seg_unit_ptr = h->seg_unit_ptr; F.segpart = h->segpart;
-  F.colsum = h->colsum; F.ticket = h->flags; F.err = h->flags + 1; F.out_state = out_state;
+  F.colsum = h->colsum; F.ticket = h->flags; F.err = h->flags + 1; F.next_chunk = h->flags + 2;
+  F.out_state = out_state;
   F.partials = partials;
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -456,7 +457,6 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
   if (ap) h->plan.kernel_adam<<<h->plan.grid, h->plan.threads, h->plan.smem_adam, stream>>>(A);
   else h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A);
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
-  h->step_parity ^= 1u;   // only a step that was enqueued consumes its counter
   if (prof && !cuda_ok(cudaEventRecord(h->ev[1], stream))) return DMX_ERR_CUDA;
   // one block per chunk-row column, one warp per segment unit. Launched as a programmatic
   // dependent of the fused pass: its blocks may become resident while that kernel drains and
@@ -474,7 +474,10 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = prof ? 0 : 1;
-  if (!cuda_ok(cudaLaunchKernelEx(&cfg, dmx::finalize_kernel, F))) return DMX_ERR_CUDA;
+  if (!cuda_ok(cudaLaunchKernelEx(&cfg, dmx::finalize_kernel, F))) {
+    (void)cudaMemsetAsync(h->flags, 0, 4 * sizeof(unsigned), stream);   // the fused pass ran: leave the handle usable
+    return DMX_ERR_CUDA;
+  }
   if (prof) {
     if (!cuda_ok(cudaEventRecord(h->ev[2], stream))) return DMX_ERR_CUDA;
     h->profiled = true;

@@ -54,8 +54,7 @@ struct StepArgs {
   int64_t P;
   int tile_group;              // R: consecutive tiles per group
   int nchunks;
-  unsigned* next_chunk;        // dynamic schedule: the counter of this step (zero at launch)
-  unsigned* next_chunk_reset;  // the counter of the following step: CTA 0 zeroes it
+  unsigned* next_chunk;        // dynamic schedule: the draw counter (zero at launch; the finalize kernel zeroes it again)
   const int64_t* seg_off;      // S+1
   const int32_t* tile_seg;     // ntiles: segment of the tile's first element; kTileBoundaryBit set
                                //         when a segment boundary lies strictly inside the tile
@@ -85,6 +84,7 @@ struct FinalArgs {
   double* colsum;              // K+4
   unsigned* ticket;
   unsigned* err;
+  unsigned* next_chunk;        // the fused pass's draw counter, zeroed here for the next step
   float* out_state;
   double* partials;            // not null: emit the raw fp64 sums of this parameter shard instead of out_state
 };
@@ -637,6 +637,7 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
       const bool internal = *reinterpret_cast<volatile unsigned*>(F.err) != 0u;
       pt[K + 4 + 2 * S] = internal ? 1.0 : 0.0;
       if (internal) *F.err = 0u;
+      *F.next_chunk = 0u;
       *F.ticket = 0u;
     }
     return;
@@ -663,6 +664,7 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
     if (internal) *F.err = 0u;
     emit_header(out, K, F.B, D, A, Qw, cs[K], cs[K + 1], bad, internal, F.adam, F.adam ? cs[K + 2] : 0.0,
                 F.adam ? cs[K + 3] : 0.0, F.P);
+    *F.next_chunk = 0u;                      // the fused pass has completed: ready for the next step (or a graph replay)
     *F.ticket = 0u;
   }
 }
@@ -841,7 +843,6 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
     uint32_t stage = 0, phase = 0, ss = 0, sphase = 0, qi = 0, qphase = 0;
     uint32_t armed_g = 0, par_g = 0, armed_s = 0, par_s = 0;   // stages armed, and the parity of the last arming
     bool ok = true;
-    if (blockIdx.x == 0 && lane == 0) *A.next_chunk_reset = 0u;   // nobody reads it before the next step
     // Lane 0 draws the next chunk a few tiles before the current chunk's copies have all been
     // issued, and fetches its descriptor when they have (the ring then holds several
     // microseconds of work, which covers that load). Drawing earlier would reserve chunks that a

@@ -101,3 +101,40 @@ def test_more_than_2_to_32_elements_closed_forms():
     assert abs(sum_m1 - (float(beta) * sum_m0 + P * c)) <= 1e-6 * P * c
     del g, params, prev, mom
     torch.cuda.empty_cache()
+
+
+def test_step_captured_in_a_cuda_graph_replays_bitwise():
+    """A step is two launches and nothing else (no allocation, no copy, no synchronisation), so
+    it can be captured in a CUDA graph; replays must give what eager steps give, bit for bit."""
+    torch, D = _torch(), _dmx()
+    wl = W.WORKLOADS[2].scaled(P=2_000_003, steps=4)
+    dp = W.DeviceProblem(wl)
+    b = dp.fill()
+    d = D.Dmx(wl.K, wl.P, dp.seg, wl.dtype)
+    out = torch.empty(d.state_len, dtype=torch.float32, device="cuda")
+    p0, m0, a0 = dp.params.clone(), dp.momentum.clone(), dp.prev_agg.clone()
+    eager = []
+    for _ in range(3):                       # the same gradients three times: the state still evolves
+        d.step(dp.grads, b, dp.params, dp.momentum, wl.lr, wl.beta, dp.prev_agg, out)
+        torch.cuda.synchronize()
+        eager.append((out.clone(), dp.params.clone(), dp.momentum.clone(), dp.prev_agg.clone()))
+    dp.params.copy_(p0); dp.momentum.copy_(m0); dp.prev_agg.copy_(a0)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            d.step(dp.grads, b, dp.params, dp.momentum, wl.lr, wl.beta, dp.prev_agg, out, stream=side.cuda_stream)
+    torch.cuda.synchronize()
+    # capture enqueues nothing: the state is still the initial one
+    assert torch.equal(dp.params, p0)
+    for i in range(3):
+        graph.replay()
+        torch.cuda.synchronize()
+        st, p, m, a = eager[i]
+        assert torch.equal(out, st) and torch.equal(dp.params, p) and torch.equal(dp.momentum, m) and torch.equal(dp.prev_agg, a), i
+    # and the handle still works eagerly after the replays
+    d.step(dp.grads, b, dp.params, dp.momentum, wl.lr, wl.beta, dp.prev_agg, out)
+    torch.cuda.synchronize()
+    assert int(out[11].item()) & 16 == 0
+    d.close()
