@@ -320,15 +320,21 @@ class DeviceProblem:
     def batch_sizes(self):
         return self.wl.batch_sizes(self.step_index)
 
-    def fill(self):
-        """Write the gradients of the current step; returns its batch sizes."""
+    def fill(self, batch=None):
+        """Write the gradients of the current step; returns its batch sizes. `batch` replaces
+        the workload's own schedule (a controller in the loop): worker k's noise then has scale
+        sigma_k / sqrt(batch[k])."""
         wl, L = self.wl, gen_lib()
-        scale = wl.grad_scale(self.step_index)
+        if batch is None:
+            scale = wl.grad_scale(self.step_index)
+        else:
+            batch = np.asarray(batch, dtype=np.int32)
+            scale = (wl.sigma() / np.sqrt(batch.astype(np.float64))).astype(np.float32)
         with self.torch.cuda.device(self.device):
             for k, g in enumerate(self.grads):
                 self._chk(L.dmxgen_grad_fill(g.data_ptr(), wl.dtype, self.mu.data_ptr(), wl.P, wl.seed, TAG_NOISE, k,
                                              self.step_index, float(scale[k]), self._stream()), "grad fill")
-        return self.batch_sizes()
+        return self.batch_sizes() if batch is None else batch
 
     def advance(self):
         self.step_index += 1

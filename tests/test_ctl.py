@@ -292,3 +292,21 @@ def test_gpu_ctl_argument_errors():
     assert call(M=0, aux=0, cols=(-1, -1, -1)) == B.OK    # no caller metrics: aux may be null
     assert call() == B.OK
     torch.cuda.synchronize()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("adam", [False, True])
+def test_gpu_closed_loop_module_runs(adam):
+    """The packaged loop (steps -> window -> decision -> batch sizes) keeps its invariants."""
+    from paper_2510_08522_b200 import closed_loop
+    recs = closed_loop.run(workload=2, P=300_011, cycles=4, k=3, hidden=16, adam=adam, sample=True, seed=3)
+    assert len(recs) == 4
+    for i, r in enumerate(recs):
+        assert r["batch"].min() >= 32 and r["batch"].max() <= 1024
+        assert np.all((r["action"] >= 0) & (r["action"] <= 4)) and np.all(np.isfinite(r["reward"]))
+        assert r["gns"] > 0 and -1.0 <= r["cos"] <= 1.0 and r["sigma_norm"] > 0
+        assert r["flags"] & 16 == 0
+        if i:
+            step = r["batch"].astype(np.int64) - recs[i - 1]["batch"]
+            want = np.clip(recs[i - 1]["batch"] + O.ACTIONS[recs[i - 1]["action"]], 32, 1024) - recs[i - 1]["batch"]
+            assert np.array_equal(step, want)
