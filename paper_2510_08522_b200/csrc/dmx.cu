@@ -463,13 +463,11 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
   // wait (griddepcontrol.wait) for its completion, which hides the launch latency between the
   // two kernels. With per-kernel timing on, the event between them needs the plain ordering.
   const int fblocks = K + 2 + 2 * F.adam + (h->nunits + dmx::kFinalWarps - 1) / dmx::kFinalWarps;
-  cudaLaunchConfig_t cfg;
-  std::memset(&cfg, 0, sizeof(cfg));
+  cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)fblocks);
   cfg.blockDim = dim3(dmx::kFinalWarps * 32);
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  std::memset(attr, 0, sizeof(attr));
+  cudaLaunchAttribute attr[1] = {};
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
