@@ -434,8 +434,10 @@ class ShardedDmx:
                 self._h = None
                 raise DmxError(rc, "dmx_create")
 
-    def step_partial(self, grads, batch_sizes, params, momentum, lr, beta, prev_agg, adam=None, stream=None):
-        """adam: None for SGD with momentum, else (second_moment, beta2, eps, t) with beta = beta1."""
+    def step_partial(self, grads, batch_sizes, params, momentum, lr, beta, prev_agg, adam=None, stream=None, local=False):
+        """adam: None for SGD with momentum, else (second_moment, beta2, eps, t) with beta = beta1.
+        local=False: every tensor has the whole problem's length and the shard works on [lo:hi);
+        local=True: every tensor holds the shard's range only (hi - lo elements, element lo first)."""
         torch = self._torch
         part = torch.zeros(self.partials_len, dtype=torch.float64, device=params.device)
         if self._h is None:                      # an empty shard contributes zeros
@@ -443,8 +445,13 @@ class ShardedDmx:
         if stream is None:
             stream = torch.cuda.current_stream(params.device).cuda_stream
         esz = 2 if self.dtype == BF16 else 4
-        gp = [g.data_ptr() + self.lo * esz for g in grads]
-        off = self.lo * 4
+        lo = 0 if local else self.lo
+        need = (self.hi - self.lo) if local else self.P
+        for x in list(grads) + [params, momentum, prev_agg]:
+            if x.numel() < need or not x.is_contiguous():
+                raise DmxError(ERR_ARG, "dmx_step_partial (tensor length)")
+        gp = [g.data_ptr() + lo * esz for g in grads]
+        off = lo * 4
         if adam is None:
             rc = dmx_step_partial(self._h, gp, batch_sizes, params.data_ptr() + off, momentum.data_ptr() + off, lr, beta,
                                   prev_agg.data_ptr() + off, part.data_ptr(), stream)

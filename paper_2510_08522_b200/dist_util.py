@@ -51,6 +51,97 @@ def allreduce_sum(t):
     return t
 
 
+def shard_ranges(P: int, world: int):
+    """[(lo, hi)] of the `world` parameter shards (the library's own split)."""
+    from . import binding as B
+    out = []
+    for r in range(world):
+        rc, lo, hi = B.dmx_shard_range(P, world, r)
+        if rc != B.OK:
+            raise B.DmxError(rc, "dmx_shard_range")
+        out.append((lo, hi))
+    return out
+
+
+def exchange_gradient_ranges(local_grad, ranges, rank: int):
+    """Worker k is rank k and holds its own gradient (P elements). Returns a (world, stride)
+    tensor whose row k holds worker k's values of THIS rank's parameter range [lo, hi) in its
+    first hi - lo entries (stride = that length rounded up to 8 elements, so that every row
+    starts on a 16-byte boundary). Every worker's values are needed, not their sum: the
+    per-worker norms and the spread across workers are computed from them. One all-to-all
+    (nccl); gloo, which has none, gathers the whole gradients and slices (tests only)."""
+    import torch
+    import torch.distributed as dist
+    world = len(ranges)
+    lo, hi = ranges[rank]
+    n = hi - lo
+    stride = (n + 7) // 8 * 8
+    out = torch.zeros((world, max(stride, 8)), dtype=local_grad.dtype, device=local_grad.device)
+    if world == 1:
+        out[0, :n] = local_grad[lo:hi]
+        return out
+    if dist.get_backend() == "nccl":
+        send = [local_grad[a:b] for a, b in ranges]
+        recv = [out[k, :n] for k in range(world)]
+        dist.all_to_all(recv, send)
+    else:
+        full = [torch.empty_like(local_grad) for _ in range(world)]
+        dist.all_gather(full, local_grad.contiguous())
+        for k in range(world):
+            out[k, :n] = full[k][lo:hi]
+    return out
+
+
+def gather_batch_sizes(b_local: int):
+    """Every worker's batch size, in rank order (host ints)."""
+    if _world <= 1:
+        return [int(b_local)]
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    mine = torch.tensor([int(b_local)], dtype=torch.int64, device=dev)
+    every = [torch.zeros_like(mine) for _ in range(_world)]
+    dist.all_gather(every, mine)
+    return [int(t.item()) for t in every]
+
+
+def allgather_ranges(shard, ranges, out_full):
+    """Rebuild a whole-length vector (the updated parameters) from the ranks' shards: out_full[lo_r:hi_r] =
+    rank r's shard. Shards differ in length, so each is padded to the longest for the collective."""
+    import torch
+    import torch.distributed as dist
+    world = len(ranges)
+    if world == 1:
+        out_full[ranges[0][0]:ranges[0][1]] = shard[:ranges[0][1] - ranges[0][0]]
+        return out_full
+    longest = max(b - a for a, b in ranges)
+    mine = torch.zeros(longest, dtype=shard.dtype, device=shard.device)
+    mine[:shard.numel()] = shard
+    every = [torch.empty_like(mine) for _ in range(world)]
+    dist.all_gather(every, mine)
+    for (a, b), t in zip(ranges, every):
+        out_full[a:b] = t[:b - a]
+    return out_full
+
+
+def worker_per_gpu_step(sh, rank, ranges, local_grad, b_local, params_shard, momentum_shard, prev_shard, lr, beta,
+                        params_full=None):
+    """One step with worker k on GPU k (K = world size) and the model state sharded by parameter
+    range: gather the batch sizes, exchange gradient ranges, run the fused pass on this rank's
+    shard (ShardedDmx `sh`, created with nshards = world, shard = rank), add the partial sums over
+    the ranks, derive the state vector (identical on every rank), and optionally rebuild the full
+    parameter vector. Returns the state vector."""
+    b = gather_batch_sizes(b_local)
+    rows = exchange_gradient_ranges(local_grad, ranges, rank)
+    part = sh.step_partial([rows[k] for k in range(len(ranges))], b, params_shard, momentum_shard, lr, beta, prev_shard,
+                           local=True)
+    allreduce_sum(part)
+    state = sh.finalize(b, part)
+    if params_full is not None:
+        allgather_ranges(params_shard, ranges, params_full)
+    return state
+
+
 def job_throughput(units_per_rank: float, local_ms: float) -> float:
     """Whole-job units per second of N replicas: N * units / slowest rank's time."""
     return _world * units_per_rank / (max_over_ranks(local_ms) * 1e-3)

@@ -67,6 +67,22 @@ WORKER = textwrap.dedent("""
     part = torch.arange(n, dtype=torch.float64) * float(hi - lo)
     DU.allreduce_sum(part)
     assert torch.equal(part, torch.arange(n, dtype=torch.float64) * float(P)), part
+    # worker k is rank k: every rank ends up with all workers' values of its own parameter range
+    Pg = 5000
+    ranges = DU.shard_ranges(Pg, world)
+    assert ranges[0][0] == 0 and ranges[-1][1] == Pg
+    grad = torch.arange(Pg, dtype=torch.float32) + 10000.0 * rank
+    rows = DU.exchange_gradient_ranges(grad, ranges, rank)
+    lo, hi = ranges[rank]
+    assert rows.shape[0] == world and rows.shape[1] %% 8 == 0 and rows.shape[1] >= hi - lo
+    for k in range(world):
+        assert torch.equal(rows[k, :hi - lo], torch.arange(lo, hi, dtype=torch.float32) + 10000.0 * k)
+        assert rows[k].data_ptr() %% 16 == 0
+    assert DU.gather_batch_sizes(32 * (rank + 1)) == [32 * (r + 1) for r in range(world)]
+    # the updated parameter shards put back together
+    full = torch.full((Pg,), -1.0)
+    DU.allgather_ranges(torch.arange(lo, hi, dtype=torch.float32) * 2.0, ranges, full)
+    assert torch.equal(full, torch.arange(Pg, dtype=torch.float32) * 2.0)
     DU.finish()
     print("rank", rank, "ok")
 """ % ROOT)
@@ -90,7 +106,7 @@ def test_partials_add_up_over_two_gloo_ranks():
 # ------------------------------------------------------------------------------------------
 # GPU: the shards of one problem, one after the other on one device, against the whole problem's oracle
 
-def _run_sharded(wl, nshards, steps, adam=False):
+def _run_sharded(wl, nshards, steps, adam=False, local=False):
     import torch
     from oracle.dmx_oracle import Oracle
     from paper_2510_08522_b200 import workload as W
@@ -111,8 +127,19 @@ def _run_sharded(wl, nshards, steps, adam=False):
             ref = orc.step(raw, b, hp, hm, wl.lr, wl.beta, hv)
         total = None
         for sh in shards:
-            part = sh.step_partial(dp.grads, b, dp.params, dp.momentum, 1e-3 if adam else wl.lr, 0.9 if adam else wl.beta,
-                                   dp.prev_agg, adam=(second, 0.999, 1e-8, t + 1) if adam else None)
+            if local:
+                # what a rank holds when worker k is GPU k: every worker's values of its own range (rows
+                # padded to 8 elements) and its own shard of the model state
+                n = sh.hi - sh.lo
+                rows = torch.zeros((wl.K, max(8, (n + 7) // 8 * 8)), dtype=dp.grads[0].dtype, device="cuda")
+                for k in range(wl.K):
+                    rows[k, :n] = dp.grads[k][sh.lo:sh.hi]
+                ps, ms, vs = (x[sh.lo:sh.hi].clone() for x in (dp.params, dp.momentum, dp.prev_agg))
+                part = sh.step_partial([rows[k] for k in range(wl.K)], b, ps, ms, wl.lr, wl.beta, vs, local=True)
+                dp.params[sh.lo:sh.hi] = ps; dp.momentum[sh.lo:sh.hi] = ms; dp.prev_agg[sh.lo:sh.hi] = vs
+            else:
+                part = sh.step_partial(dp.grads, b, dp.params, dp.momentum, 1e-3 if adam else wl.lr, 0.9 if adam else wl.beta,
+                                       dp.prev_agg, adam=(second, 0.999, 1e-8, t + 1) if adam else None)
             total = part if total is None else total + part
         st = shards[0].finalize(b, total, adam=adam)
         torch.cuda.synchronize()
@@ -141,6 +168,38 @@ def _run_sharded(wl, nshards, steps, adam=False):
 def test_gpu_shards_match_the_whole_problem_oracle(idx, P, nshards):
     from paper_2510_08522_b200 import workload as W
     _run_sharded(W.WORKLOADS[idx].scaled(P=P, steps=3), nshards, 3)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("idx,P,nshards", [(1, 333_337, 3), (4, 523_777, 4)])
+def test_gpu_shards_with_rank_local_buffers(idx, P, nshards):
+    from paper_2510_08522_b200 import workload as W
+    _run_sharded(W.WORKLOADS[idx].scaled(P=P, steps=2), nshards, 2, local=True)
+
+
+@pytest.mark.gpu
+def test_gpu_worker_per_gpu_step_on_one_rank():
+    """The packaged multi-GPU step with a world of one: K = 1 worker, one shard."""
+    import torch
+    from oracle.dmx_oracle import Oracle
+    from paper_2510_08522_b200 import dist_util as DU
+    P = 70_001
+    rng = np.random.default_rng(9)
+    g = rng.normal(size=P).astype(np.float32)
+    p0 = rng.normal(scale=0.05, size=P).astype(np.float32)
+    seg = [0, 1000, P]
+    DU.init(1)
+    ranges = DU.shard_ranges(P, 1)
+    sh = D.ShardedDmx(1, P, seg, B.F32, 1, 0)
+    tp, tm, tv = torch.from_numpy(p0.copy()).cuda(), torch.zeros(P, device="cuda"), torch.zeros(P, device="cuda")
+    full = torch.empty(P, device="cuda")
+    st = DU.worker_per_gpu_step(sh, 0, ranges, torch.from_numpy(g).cuda(), 64, tp, tm, tv, 0.1, 0.9, params_full=full)
+    torch.cuda.synchronize()
+    hp, hm, hv = p0.copy(), np.zeros(P, np.float32), np.zeros(P, np.float32)
+    ref = Oracle(1, P, seg, 0).step([g], [64], hp, hm, 0.1, 0.9, hv)
+    assert np.allclose(st.cpu().numpy(), ref, rtol=1e-4, atol=1e-7)
+    assert np.allclose(full.cpu().numpy(), hp, rtol=1e-6, atol=1e-8) and np.allclose(tm.cpu().numpy(), hm, rtol=1e-6, atol=1e-8)
+    sh.close()
 
 
 @pytest.mark.gpu
