@@ -72,3 +72,25 @@ def test_plan_rejects_bad_arguments():
     assert D.dmx_plan_chunks(10, 4, 7, 896, 148)[0] == B.ERR_ARG
     assert D.dmx_plan_chunks(10, 4, B.F32, 0, 148)[0] == B.ERR_ARG
     assert D.dmx_plan_chunks(10, 4, B.F32, 896, 0)[0] == B.ERR_ARG
+
+
+def test_random_problems_are_always_tiled_exactly():
+    hyp = pytest.importorskip("hypothesis")
+    st = hyp.strategies
+
+    @hyp.settings(max_examples=150, deadline=None)
+    @hyp.given(P=st.integers(1, 60_000_000), K=st.integers(1, 64), dtype=st.sampled_from([B.F32, B.BF16]),
+               ctas=st.integers(1, 320))
+    def check(P, K, dtype, ctas):
+        tile = 896 if dtype == B.F32 else 1792
+        n, t0, nt, stv, R, grid = D.dmx_plan_chunks(P, K, dtype, tile, ctas)
+        ntiles = -(-P // tile)
+        assert n > 0 and 1 <= grid <= ctas and sum(nt) == ntiles and max(nt) <= 32
+        seen = np.zeros(ntiles, dtype=np.int32)
+        for c in range(n):
+            np.add.at(seen, tiles_of(t0[c], nt[c], stv[c], R), 1)
+        assert np.all(seen == 1)
+        if P % tile:
+            assert tiles_of(t0[0], nt[0], stv[0], R)[-1] == ntiles - 1
+
+    check()
