@@ -126,7 +126,7 @@ def step_bytes(wl, optimizer):
 L2_FLUSH_BELOW = 4 << 30      # workloads streaming less than this per step get an L2 flush between steps
 
 
-def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profile=True, optimizer="sgd"):
+def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profile=True, optimizer="sgd", sustained=True):
     """Time `steps` steps of workload `wl` on `device`. Returns a dict of local measurements.
     Workloads whose step streams only a few times the L2's size get a 512 MB write between the
     (untimed) input generation and the timed step, so that no step starts on a warm L2."""
@@ -210,7 +210,7 @@ def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profi
         res["d2h_bytes"] = d.state_len * 4
         res["e2e_launches"] = e2e_steps * d.launches_per_step
         del host
-    if sample_clocks and world_is_one() and optimizer == "sgd":
+    if sustained and sample_clocks and world_is_one() and optimizer == "sgd":
         # the same step launched back to back for about a second on one set of gradients (inputs far larger
         # than L2): the duty cycle of the timed loop above is low (input generation sits between its steps);
         # at full duty the board reaches its power limit and the SM clock drops, which this path feels
@@ -288,6 +288,8 @@ def main():
                     help="1: also time the remaining workloads briefly and list them under 'workloads' (N=1 only)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-sample-elems", type=int, default=128 << 20, help="0: skip the CPU-baseline leg")
+    ap.add_argument("--sustained", type=int, default=1,
+                    help="1: after the timed steps, also launch the step back to back for about a second (N=1 only)")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "adam"],
                     help="update applied by the step (the metric's workload uses sgd)")
     ap.add_argument("--P", type=int, default=0, help="run the workload's structure at another size (profiling captures)")
@@ -337,7 +339,8 @@ def main():
     DU.init(world, "nccl")
     DU.barrier()
     torch.cuda.synchronize()
-    res = run_workload(wl, args.steps, args.warmup, device, args.e2e_steps, optimizer=args.optimizer)
+    res = run_workload(wl, args.steps, args.warmup, device, args.e2e_steps, optimizer=args.optimizer,
+                       sustained=bool(args.sustained))
     torch.cuda.synchronize()
     DU.barrier()
     total_ms = DU.max_over_ranks(res["total_ms"])
