@@ -100,17 +100,22 @@ Plan pick_direct(int K) {
 
 // Pipelined (bulk-copy ring) kernels. Ring geometry: 7 consumer warps + the producer warp = 8
 // warps, so that a thread may use up to 255 registers (9 warps are allocated as 12 and cap it
-// at 168, which spilled at K = 32); 4 gradient streams per 14 KB stage (smaller stages lose to
-// the per-stage synchronisation, larger ones leave too few in flight).
+// at 168, which spilled at K = 32). A stage holds up to 16 gradient streams (56 KB): the
+// consumers pay one wait, one release and one batch of shared-memory loads per stage, and with
+// 4 streams per stage that per-stage work made the consumers the limiter as soon as the SM
+// clock dropped under the board's power limit (steps launched back to back: 5.8 -> 6.5 TB/s at
+// K = 32 bf16, 6.2 -> 6.8 TB/s at K = 32 fp32 with 16; the time at full clock is unchanged).
+// Stages smaller than 4 streams lose even at full clock.
 // The producer runs at most NSS tiles ahead of the consumers (a tile's state stage is freed when
 // the consumers have read it), so the bytes in flight per SM are min(ring, NSS tiles). With many
-// workers one tile already fills the ring and one state stage is best (a second one measured 2-3 %
-// slower at K = 32); with few workers a tile is small, and one state stage left only ~40 KB per
-// SM in flight (0.76 of the copy rate at K = 8): there the ring is split into as many whole tiles
-// (gradient stages + a state stage each) as fit.
+// workers one tile already fills the ring and one state stage is enough; with few workers a tile
+// is small, and one state stage left only ~40 KB per SM in flight (0.76 of the copy rate at
+// K = 8): there the ring is split into as many whole tiles (gradient stages + a state stage
+// each) as fit.
 template <int KT, bool BF16, bool ADAM>
 struct Ring {
-  static constexpr int CW = 7, G = 4;
+  static constexpr int CW = 7;
+  static constexpr int G = KT < 16 ? KT : 16;                                       // gradient streams per stage
   static constexpr int kStage = CW * 32 * 16 * G;                                   // bytes of a gradient stage
   static constexpr int kState = CW * 32 * (BF16 ? 8 : 4) * 4 * (ADAM ? 4 : 3);      // bytes of a state stage
   static constexpr int kTile = (KT + G - 1) / G * kStage + kState;                  // shared memory of one tile
@@ -118,8 +123,8 @@ struct Ring {
   static constexpr int NSS = kAhead < 1 ? 1 : (kAhead > 8 ? 8 : kAhead);
   static constexpr int kRed = (int)((sizeof(dmx::RedArea<KT, CW>) + 15) / 16 * 16);
   static constexpr int kFit = (227 * 1024 - NSS * (kState + 16) - kRed - 128) / (kStage + 16);
-  static constexpr int kTuned = BF16 ? (ADAM ? 12 : 13) : 14;                       // measured best with one state stage
-  static constexpr int NSTAGE = NSS == 1 ? kTuned : (kFit > 32 ? 32 : kFit);
+  static constexpr int NSTAGE = kFit > 32 ? 32 : kFit;
+  static_assert(NSTAGE >= 2, "the ring needs two gradient stages");
   typedef dmx::PipeCfg<KT, BF16, CW, G, NSTAGE, NSS, ADAM> Cfg;
 };
 
