@@ -85,3 +85,16 @@ def test_philox_known_answer():
     assert [int(x) for x in r] == [0x408f276d, 0x41c83b0e, 0xa20bc7c6, 0x6d5451fd]
     r = W.philox4x32(0x243f6a88, 0x85a308d3, 0x13198a2e, 0x03707344, 0xa4093822, 0x299f31d0)
     assert [int(x) for x in r] == [0xd16cfe09, 0x94fdcceb, 0x5001e420, 0x24126ea1]
+
+
+def test_header_compiles_as_plain_c(tmp_path):
+    # the boundary is a C ABI: the header must be valid C99 on its own (no C++, no CUDA types)
+    import subprocess
+    src = tmp_path / "use_dmx.c"
+    src.write_text('#include "dmx.h"\n'
+                   'int use(void) { dmx_handle* h = 0; int64_t seg[2] = {0, 8};\n'
+                   '  int rc = dmx_create(2, 8, seg, 1, DMX_F32, &h);\n'
+                   '  return rc == DMX_OK ? dmx_state_len(h) + DMX_ST_HDR + DMX_FLAG_INTERNAL + DMX_CTL_ACTIONS : rc; }\n')
+    r = subprocess.run(["gcc", "-std=c99", "-pedantic", "-Wall", "-Werror", "-fsyntax-only", "-I", os.path.join(ROOT, "include"), str(src)],
+                       capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
