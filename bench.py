@@ -52,7 +52,7 @@ def recorded_traffic(workload_name):
     """DRAM bytes per launch of the fused kernel from the committed ncu capture, if the
     kernel sources are still the ones that were captured; else None."""
     try:
-        with open(os.path.join(ROOT, "profiles", "ncu_traffic.json")) as f:
+        with open(os.path.join(ROOT, "profiles", "pipe_kernel_dram_traffic.json")) as f:
             rec = json.load(f)
         if rec.get("kernel_source_digest") != kernel_source_digest():
             return None
