@@ -138,3 +138,28 @@ def test_step_captured_in_a_cuda_graph_replays_bitwise():
     torch.cuda.synchronize()
     assert int(out[11].item()) & 16 == 0
     d.close()
+
+
+@pytest.mark.parametrize("idx", [3, 4])
+def test_full_size_step_is_bitwise_reproducible_under_the_dynamic_schedule(idx):
+    """At full size every CTA draws dozens of chunks and which CTA gets which varies from run to
+    run; the results must not."""
+    torch, D = _torch(), _dmx()
+    wl = W.WORKLOADS[idx]
+    dp = W.DeviceProblem(wl)
+    b = dp.fill()
+    dp.prev_agg.normal_(0, 0.05)                     # a non-trivial previous aggregate
+    p0, m0, a0 = dp.params.clone(), dp.momentum.clone(), dp.prev_agg.clone()
+    d = D.Dmx(wl.K, wl.P, dp.seg, wl.dtype)
+    runs = []
+    for _ in range(3):
+        dp.params.copy_(p0); dp.momentum.copy_(m0); dp.prev_agg.copy_(a0)
+        st = d.step(dp.grads, b, dp.params, dp.momentum, wl.lr, wl.beta, dp.prev_agg)
+        torch.cuda.synchronize()
+        runs.append((st.clone(), dp.params.clone(), dp.momentum.clone(), dp.prev_agg.clone()))
+        if len(runs) > 1:
+            for x, y in zip(runs[0], runs[-1]):
+                assert torch.equal(x, y)
+            runs.pop()
+    assert int(runs[0][0][11].item()) & 16 == 0
+    d.close()
