@@ -389,3 +389,37 @@ def test_unbiasedness_with_per_worker_noise_scales():
     expect = wl.P * float(np.sum(sig ** 2 * (1 - w))) / (wl.K - 1)
     assert abs(r["st"][ST["TRS"]] / expect - 1.0) < 0.02
     assert 0.5 <= sig.min() and sig.max() <= 2.0 and 16 <= b.min() and b.max() <= 1024
+
+
+def _seeded_golden():
+    import json
+    with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "seeded_small_k3.json")) as f:
+        return json.load(f)
+
+
+def test_seeded_golden_is_what_the_oracle_computes_and_its_exact_parts_check_by_hand():
+    """The stored fixture (written by tests/golden/make_seeded_golden.py) still equals the oracle's
+    output, and the parts of it that are exact rationals are recomputed here with Python
+    fractions from the definitions."""
+    from fractions import Fraction as Fr
+    d = _seeded_golden()
+    K, P, seg, b = d["K"], d["P"], d["seg_offsets"], d["batch_sizes"]
+    grads = [np.array(g, np.float32) for g in d["grads"]]
+    params, mom, prev = (np.array(d[k], np.float32) for k in ("params", "momentum", "prev_agg"))
+    prev_in = prev.copy()
+    st = Oracle(K, P, seg, 0).step(grads, b, params, mom, d["lr"], d["beta"], prev)
+    assert [float(v) for v in st] == d["expect"]["state"]
+    assert prev.tolist() == d["expect"]["agg"] and mom.tolist() == d["expect"]["momentum"] and params.tolist() == d["expect"]["params"]
+    B = sum(b)
+    g = [sum(Fr(b[k]) * Fr(float(grads[k][j])) for k in range(K)) / B for j in range(P)]
+    assert [float(x) for x in g] == d["expect"]["agg"]
+    A = sum(x * x for x in g)
+    D = sum(Fr(b[k]) * (Fr(float(grads[k][j])) - g[j]) ** 2 for k in range(K) for j in range(P))
+    assert float(A) == d["expect"]["state"][1] and float(D / (K - 1)) == d["expect"]["state"][2]
+    assert float(A - D / (K - 1) / B) == d["expect"]["state"][3]
+    assert float(sum(g[j] * Fr(float(prev_in[j])) for j in range(P))) == d["expect"]["state"][6]
+    S = len(seg) - 1
+    for s in range(S):
+        Vs = sum(Fr(b[k]) * (Fr(float(grads[k][j])) - g[j]) ** 2 for k in range(K) for j in range(seg[s], seg[s + 1])) / (K - 1)
+        assert float(Vs) == d["expect"]["state"][16 + K + s]
+        assert float(sum(g[j] ** 2 for j in range(seg[s], seg[s + 1]))) == d["expect"]["state"][16 + K + S + s]
