@@ -183,3 +183,43 @@ def test_gpu_matches_the_stored_seeded_golden():
     # integer-valued inputs with B = 8: the aggregate and the update are exact in fp32 too
     assert prev.cpu().tolist() == exp["agg"] and mom.cpu().tolist() == exp["momentum"] and params.cpu().tolist() == exp["params"]
     assert np.allclose(st.cpu().numpy(), np.array(exp["state"]), rtol=1e-6, atol=1e-6)
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_step_from_host_gradients_equals_the_device_step(dtype):
+    """dmx_step_host: gradients in pinned host memory, staged by the call; same result, bit for bit,
+    as dmx_step on the same values, and the state vector arrives in host memory."""
+    torch, D = _torch(), _dmx()
+    from paper_2510_08522_b200 import binding as B
+    K, P = 5, 300_007
+    seg = [0, 1000, 150_000, P]
+    rng = np.random.default_rng(21)
+    gdt = torch.float32 if dtype == 0 else torch.bfloat16
+    host = [torch.from_numpy(rng.normal(size=P).astype(np.float32)).to(gdt).pin_memory() for _ in range(K)]
+    b = [32, 64, 16, 128, 256]
+    p0 = torch.from_numpy(rng.normal(scale=0.05, size=P).astype(np.float32)).cuda()
+    m0 = torch.from_numpy(rng.normal(scale=0.01, size=P).astype(np.float32)).cuda()
+    a0 = torch.from_numpy(rng.normal(scale=0.1, size=P).astype(np.float32)).cuda()
+    d = D.Dmx(K, P, seg, dtype)
+    # reference: copy by hand, then the device step
+    dev = [h.cuda() for h in host]
+    p1, m1, a1 = p0.clone(), m0.clone(), a0.clone()
+    st_ref = d.step(dev, b, p1, m1, 0.1, 0.9, a1).clone()
+    # the host form
+    staging = [torch.empty(P, dtype=gdt, device="cuda") for _ in range(K)]
+    p2, m2, a2 = p0.clone(), m0.clone(), a0.clone()
+    out_dev = torch.empty(d.state_len, dtype=torch.float32, device="cuda")
+    out_host = torch.zeros(d.state_len, dtype=torch.float32).pin_memory()
+    d.step_host(host, staging, b, p2, m2, 0.1, 0.9, a2, out_dev, out_host)       # synchronous
+    assert torch.equal(out_host, st_ref.cpu()) and torch.equal(out_dev, st_ref)
+    assert torch.equal(p1, p2) and torch.equal(m1, m2) and torch.equal(a1, a2)
+    for s, h in zip(staging, host):
+        assert torch.equal(s.cpu(), h)
+    # argument errors come back as codes
+    hp = [h.data_ptr() for h in host]
+    sp = [s.data_ptr() for s in staging]
+    args = (b, p2.data_ptr(), m2.data_ptr(), 0.1, 0.9, a2.data_ptr(), out_dev.data_ptr(), out_host.data_ptr())
+    assert B.dmx_step_host(d._h, hp, [sp[0] + 2] + sp[1:], *args) == B.ERR_ALIGN
+    assert B.dmx_step_host(d._h, hp, sp, b, p2.data_ptr(), m2.data_ptr(), 0.1, 0.9, a2.data_ptr(), out_dev.data_ptr(), 0) == B.ERR_ARG
+    assert B.dmx_step_host(None, hp, sp, *args) == B.ERR_HANDLE
+    d.close()
