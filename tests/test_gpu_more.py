@@ -223,3 +223,26 @@ def test_step_from_host_gradients_equals_the_device_step(dtype):
     assert B.dmx_step_host(d._h, hp, sp, b, p2.data_ptr(), m2.data_ptr(), 0.1, 0.9, a2.data_ptr(), out_dev.data_ptr(), 0) == B.ERR_ARG
     assert B.dmx_step_host(None, hp, sp, *args) == B.ERR_HANDLE
     d.close()
+
+
+def test_profiling_hooks():
+    torch, D = _torch(), _dmx()
+    from paper_2510_08522_b200 import binding as B
+    c = Custom(rnd(3, 4, 50_000), [32, 64, 96, 128], [0, 50_000])
+    d = D.Dmx(c.K, c.P, c.seg, 0)
+    assert d.launches_per_step == 2 and B.dmx_launches_per_step(None) == B.ERR_HANDLE
+    assert B.dmx_get_profile(d._h)[0] == B.ERR_ARG            # profiling is off
+    d.set_profiling(True)
+    assert B.dmx_get_profile(d._h)[0] == B.ERR_ARG            # on, but no step recorded yet
+    st_on = d.step(c.d_grads, c.b, c.d_params, c.d_momentum, 0.1, 0.9, c.d_prev).clone()
+    fused_ms, fin_ms = d.profile()
+    assert 0.0 < fused_ms < 50.0 and 0.0 < fin_ms < 50.0
+    d.set_profiling(False)
+    assert B.dmx_get_profile(d._h)[0] == B.ERR_ARG
+    # timing on or off does not change results: rerun the same step from the same state without it
+    c2 = Custom(rnd(3, 4, 50_000), [32, 64, 96, 128], [0, 50_000])
+    st_off = d.step(c2.d_grads, c2.b, c2.d_params, c2.d_momentum, 0.1, 0.9, c2.d_prev)
+    torch.cuda.synchronize()
+    assert torch.equal(st_on, st_off) and torch.equal(c.d_params, c2.d_params)
+    assert B.dmx_set_profiling(None, 1) == B.ERR_HANDLE and B.dmx_last_cuda_error() == 0
+    d.close()
