@@ -246,3 +246,44 @@ def test_profiling_hooks():
     assert torch.equal(st_on, st_off) and torch.equal(c.d_params, c2.d_params)
     assert B.dmx_set_profiling(None, 1) == B.ERR_HANDLE and B.dmx_last_cuda_error() == 0
     d.close()
+
+
+@pytest.mark.parametrize("seed", [11, 12])
+def test_random_problems_match_the_oracle(seed):
+    """Seeded random problems: K from 1 to 64 around the kernel table's capacities, P around the
+    tile sizes and up to a few hundred tiles, random segment tables, both gradient types, both
+    updates, sometimes with odd scheduling knobs."""
+    torch, D = _torch(), _dmx()
+    rng = np.random.default_rng(seed)
+    for case in range(60):
+        K = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 9, 15, 16, 17, 31, 32, 33, 48, 64]))
+        P = int(rng.choice([1, 7, 895, 896, 897, 1792, 1793, int(rng.integers(1, 5000)), int(rng.integers(5000, 400_000))]))
+        dtype = int(rng.integers(0, 2))
+        S = int(rng.choice([1, 2, 3, 17, 200])) if P > 1 else 1
+        seg = [0] + sorted(int(v) for v in rng.integers(0, P + 1, S - 1)) + [P]
+        b = [int(v) for v in rng.choice([1, 16, 32, 33, 64, 100, 256, 1024], K)]
+        knobs = {}
+        if rng.random() < 0.3:
+            knobs = dict(DMX_CHUNK_TILES=int(rng.choice([1, 2, 5, 8, 33])), DMX_TILE_GROUP=int(rng.choice([1, 2, 3, 4])))
+        adam = rng.random() < 0.3
+        mu = 0.1 * rng.standard_normal(P)
+        g32 = [(mu + rng.standard_normal(P) / np.sqrt(b[k])).astype(np.float32) for k in range(K)]
+        what = "case %d: K=%d P=%d dtype=%d S=%d adam=%s knobs=%s" % (case, K, P, dtype, S, adam, knobs)
+        with env(**knobs):
+            c = Custom(g32, b, seg, dtype, params=0.05 * rng.standard_normal(P), momentum=0.01 * rng.standard_normal(P),
+                       prev=0.1 * rng.standard_normal(P))
+            if not adam:
+                st, _, _ = c.run(what=what)
+                assert int(st[11]) & 16 == 0, what
+                continue
+            h2 = np.abs(0.01 * rng.standard_normal(P)).astype(np.float32)
+            d2 = torch.from_numpy(h2.copy()).cuda()
+            conds = PT.cond_vectors_adam(c.wide, c.b, c.params, c.momentum, h2, 1e-3, 0.9, 0.999, 1e-8, 3)
+            Oracle(K, P, c.seg, dtype).step_adam(c.raw, c.b, c.params, c.momentum, h2, 1e-3, 0.9, 0.999, 1e-8, 3, c.prev)
+            d = D.Dmx(K, P, c.seg, dtype)
+            st = d.step_adam(c.d_grads, c.b, c.d_params, c.d_momentum, d2, 1e-3, 0.9, 0.999, 1e-8, 3, c.d_prev)
+            torch.cuda.synchronize()
+            d.close()
+            PT.check_vectors_adam(dtype, (c.d_prev.cpu().numpy(), c.d_momentum.cpu().numpy(), d2.cpu().numpy(), c.d_params.cpu().numpy()),
+                                  (c.prev, c.momentum, h2, c.params), conds, what)
+            assert int(st[11].item()) & 16 == 0, what
