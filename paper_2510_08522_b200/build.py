@@ -19,7 +19,7 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
               "-shared", "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 
 TARGETS = {
-    "libdmx.so": (["dmx.cu", "dmx_static.cu", "dmx_agg.cu", "dmx_ctl.cu"], ["dmx_kernels.cuh", os.path.join(INCLUDE, "dmx.h")]),
+    "libdmx.so": (["dmx.cu", "dmx_static.cu", "dmx_agg.cu", "dmx_ctl.cu"], ["dmx_kernels.cuh", "dmx_host.h", os.path.join(INCLUDE, "dmx.h")]),
     "libdmx_gen.so": (["dmx_gen.cu"], []),
 }
 

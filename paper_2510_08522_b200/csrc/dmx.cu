@@ -9,11 +9,14 @@
 #include <new>
 #include <vector>
 
+#include "dmx_host.h"
 #include "dmx_kernels.cuh"
 
 namespace {
-
 thread_local int g_last_cuda = 0;
+}
+
+namespace dmxh {
 
 bool cuda_ok(cudaError_t e) {
   if (e == cudaSuccess) return true;
@@ -21,6 +24,69 @@ bool cuda_ok(cudaError_t e) {
   (void)cudaGetLastError();
   return false;
 }
+
+static bool overlap(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
+  return x < y + nb && y < x + na;
+}
+
+int check_step_buffers(int K, int64_t P, int grad_dtype, const StepBuffers& sb, int64_t* B, int* pivot) {
+  if (!sb.grad_ptrs || !sb.batch_sizes || !sb.params || !sb.momentum || !sb.prev_agg || !sb.out) return DMX_ERR_ARG;
+  const size_t gbytes = (size_t)P * (grad_dtype == DMX_BF16 ? 2 : 4), sbytes = (size_t)P * 4;
+  *B = 0;
+  *pivot = 0;
+  for (int k = 0; k < K; ++k) {
+    if (!sb.grad_ptrs[k]) return DMX_ERR_ARG;
+    if (sb.batch_sizes[k] < 1) return DMX_ERR_BATCH;
+    *B += sb.batch_sizes[k];
+    if (sb.batch_sizes[k] > sb.batch_sizes[*pivot]) *pivot = k;
+  }
+  for (int k = 0; k < K; ++k)
+    if ((uintptr_t)sb.grad_ptrs[k] & 15) return DMX_ERR_ALIGN;
+  if (((uintptr_t)sb.params & 15) || ((uintptr_t)sb.momentum & 15) || ((uintptr_t)sb.prev_agg & 15) ||
+      ((uintptr_t)sb.out & sb.out_align_mask) || ((uintptr_t)sb.second & 15))
+    return DMX_ERR_ALIGN;
+  const void* st[5] = {sb.params, sb.momentum, sb.prev_agg, sb.out, sb.second};
+  const size_t sn[5] = {sbytes, sbytes, sbytes, sb.out_bytes, sbytes};
+  const int nst = sb.second ? 5 : 4;
+  for (int i = 0; i < nst; ++i) {
+    for (int j = i + 1; j < nst; ++j)
+      if (overlap(st[i], sn[i], st[j], sn[j])) return DMX_ERR_ARG;
+    for (int k = 0; k < K; ++k)
+      if (overlap(st[i], sn[i], sb.grad_ptrs[k], gbytes)) return DMX_ERR_ARG;
+  }
+  return DMX_OK;
+}
+
+void pack_workers(int K, const void* const* grad_ptrs, const int32_t* batch_sizes, int pivot, int64_t B, float lr,
+                  float beta, dmx::StepArgs& A, int* orig, double* b) {
+  int slot = 0;
+  for (int i = -1; i < K; ++i) {
+    const int k = i < 0 ? pivot : i;
+    if (i >= 0 && k == pivot) continue;
+    A.grad[slot] = grad_ptrs[k];
+    A.w[slot] = (float)((double)batch_sizes[k] / (double)B);
+    A.bf[slot] = (float)batch_sizes[k];
+    A.bd[slot] = (double)batch_sizes[k];
+    orig[slot] = k;
+    b[slot] = (double)batch_sizes[k];
+    ++slot;
+  }
+  A.lr = lr; A.beta = beta; A.Bf = (float)B;
+  A.rB = 1.0 / (double)B; A.lr64 = (double)lr; A.beta64 = (double)beta;
+}
+
+int check_current_device(int device) {
+  int cur = -1;
+  if (!cuda_ok(cudaGetDevice(&cur))) return DMX_ERR_CUDA;
+  return cur == device ? DMX_OK : DMX_ERR_HANDLE;
+}
+
+}  // namespace dmxh
+
+namespace {
+
+using dmxh::cuda_ok;
 
 constexpr uint64_t kMagic = 0x444d585f48414e44ull;  // "DMX_HAND"
 
@@ -229,11 +295,6 @@ void free_handle(dmx_handle* h) {
   delete h;
 }
 
-bool overlap(const void* a, size_t na, const void* b, size_t nb) {
-  const uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
-  return x < y + nb && y < x + na;
-}
-
 }  // namespace
 
 extern "C" {
@@ -380,38 +441,22 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
               const AdamParams* ap, double* partials = nullptr) {
   // `partials` (a parameter shard of a larger problem): the raw sums go there and out_state is not written
   if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
-  if (!grad_ptrs || !batch_sizes || !params || !momentum || !prev_agg || (!out_state && !partials)) return DMX_ERR_ARG;
+  if (!out_state && !partials) return DMX_ERR_ARG;
   if (ap && (!ap->second || ap->t < 1 || !(beta >= 0.f && beta < 1.f) || !(ap->beta2 >= 0.f && ap->beta2 < 1.f) ||
              !(ap->eps >= 0.f)))
     return DMX_ERR_ARG;
   const int K = h->K;
-  const size_t esz = h->dtype == DMX_BF16 ? 2 : 4;
-  const size_t gbytes = (size_t)h->P * esz, sbytes = (size_t)h->P * 4;
-  const size_t obytes = partials ? (size_t)(K + 5 + 2 * h->S) * 8 : (size_t)(DMX_ST_HDR + K + 2 * h->S) * 4;
-  const void* outp = partials ? (const void*)partials : (const void*)out_state;
+  dmxh::StepBuffers sb = {grad_ptrs, batch_sizes, params, momentum, prev_agg, ap ? ap->second : nullptr,
+                          partials ? (const void*)partials : (const void*)out_state,
+                          partials ? (size_t)(K + 5 + 2 * h->S) * 8 : (size_t)(DMX_ST_HDR + K + 2 * h->S) * 4,
+                          partials ? 7u : 3u};
   int64_t B = 0;
   int pivot = 0;
-  for (int k = 0; k < K; ++k) {
-    if (!grad_ptrs[k]) return DMX_ERR_ARG;
-    if (batch_sizes[k] < 1) return DMX_ERR_BATCH;
-    B += batch_sizes[k];
-    if (batch_sizes[k] > batch_sizes[pivot]) pivot = k;
-  }
-  for (int k = 0; k < K; ++k)
-    if ((uintptr_t)grad_ptrs[k] & 15) return DMX_ERR_ALIGN;
-  if (((uintptr_t)params & 15) || ((uintptr_t)momentum & 15) || ((uintptr_t)prev_agg & 15) ||
-      ((uintptr_t)outp & (partials ? 7 : 3)))
-    return DMX_ERR_ALIGN;
-  if (ap && ((uintptr_t)ap->second & 15)) return DMX_ERR_ALIGN;
-  const void* st[5] = {params, momentum, prev_agg, outp, ap ? ap->second : nullptr};
-  const size_t sn[5] = {sbytes, sbytes, sbytes, obytes, sbytes};
-  const int nst = ap ? 5 : 4;
-  for (int i = 0; i < nst; ++i) {
-    for (int j = i + 1; j < nst; ++j)
-      if (overlap(st[i], sn[i], st[j], sn[j])) return DMX_ERR_ARG;
-    for (int k = 0; k < K; ++k)
-      if (overlap(st[i], sn[i], grad_ptrs[k], gbytes)) return DMX_ERR_ARG;
-  }
+  int rc = dmxh::check_step_buffers(K, h->P, h->dtype, sb, &B, &pivot);
+  if (rc != DMX_OK) return rc;
+  // the handle's tables and scratch live on the device that was current in dmx_create
+  rc = dmxh::check_current_device(h->device);
+  if (rc != DMX_OK) return rc;
 
   dmx::StepArgs A;
   dmx::FinalArgs F;
@@ -419,19 +464,8 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
   std::memset(&F, 0, sizeof(F));
   // processing order: the worker with the largest batch first (the pivot), the others in
   // the caller's order
-  int slot = 0;
-  for (int i = -1; i < K; ++i) {
-    const int k = i < 0 ? pivot : i;
-    if (i >= 0 && k == pivot) continue;
-    A.grad[slot] = grad_ptrs[k];
-    A.w[slot] = (float)((double)batch_sizes[k] / (double)B);
-    A.bf[slot] = (float)batch_sizes[k];
-    F.orig[slot] = k;
-    F.b[slot] = (double)batch_sizes[k];
-    ++slot;
-  }
+  dmxh::pack_workers(K, grad_ptrs, batch_sizes, pivot, B, lr, beta, A, F.orig, F.b);
   A.params = params; A.momentum = momentum; A.prev = prev_agg;
-  A.lr = lr; A.beta = beta; A.Bf = (float)B;
   if (ap) {
     // bias corrections in fp64 from the fp32 coefficients, handed over as fp32 factors
     A.second = ap->second; A.beta2 = ap->beta2; A.eps = ap->eps;

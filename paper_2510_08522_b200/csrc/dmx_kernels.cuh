@@ -13,6 +13,16 @@
 // cancellation is between noise-sized terms only. The arithmetic runs on pairs of fp32
 // values with the packed f32x2 instructions of sm_100 (each lane IEEE fp32, round to nearest).
 //
+// With fp32 gradients the per-parameter recurrence itself (aggregate -> momentum -> parameter) is
+// carried in fp64 and rounded once at each store, as its definition says:
+//   g = (sum_k b_k x_k) / B,  m' = beta m + g,  theta' = theta - lr m'.
+// The stored fp32 values are then the correctly rounded ones in all but about one case in 2^29,
+// so a long run stays on the trajectory of the definition bit for bit; with an fp32 aggregate
+// every step left a last-bit difference in g that the momentum's and the parameters' own
+// roundings turned into whole-ulp differences, amplified by 1/(1 - beta) and accumulated over
+// the steps (1e-4 of a parameter's forward-error scale after 100 steps). The statistics keep
+// the fp32 shifted sums. With bf16 gradients (tolerance 4e-3) the aggregate stays fp32.
+//
 // Work layout. The parameter range is cut into tiles of T elements, taken in groups of R
 // consecutive tiles. The unit of work is a chunk: a few groups, interleaved with the other
 // chunks of its wave (chunk l of a wave of n chunks holds groups first+l, first+l+n, ...), so
@@ -44,6 +54,8 @@ struct StepArgs {
   const void* grad[kMaxK];
   float w[kMaxK];        // b_k / B
   float bf[kMaxK];       // b_k
+  double bd[kMaxK];      // b_k (fp32 gradients: the fp64 aggregate)
+  double rB, lr64, beta64;   // 1/B, and lr and beta widened exactly
   float* params;
   float* momentum;
   float* prev;
@@ -163,7 +175,9 @@ __device__ __forceinline__ void st_stream(float* p, float a, float b, float c, f
 template <int KT, int VEC>
 struct Acc {
   static constexpr int NP2 = VEC / 2;
+  static constexpr bool WIDE = VEC == 4;   // fp32 gradients (4 per 16 bytes): aggregate and update in fp64
   u64 np[NP2], s1[NP2], s2[NP2];    // -pivot, sum w e, sum b e^2 (pairs)
+  double S[WIDE ? VEC : 1];         // sum_k b_k x_k (exact products, fp64 sums)
   float q[KT];                      // per-worker sum of squares (chunk)
   float c, pp, vs, ns;              // <g,a>, |a|^2, current segment's V and N partials
   float su, su2;                    // Adam only: sums of g/(sqrt(vhat)+eps) and of its square (chunk)
@@ -175,10 +189,19 @@ struct Acc {
     su = su2 = 0.f;
   }
   // k is a compile-time constant after unrolling at every call site, so q[k] is a register.
-  __device__ __forceinline__ void add(int k, const u64* x, float w, float bf) {
+  __device__ __forceinline__ void add(int k, const u64* x, float w, float bf, double bd) {
     u64 sq = mul2(x[0], x[0]);
 #pragma unroll
     for (int i = 1; i < NP2; ++i) sq = fma2(x[i], x[i], sq);
+    if constexpr (WIDE) {
+#pragma unroll
+      for (int i = 0; i < NP2; ++i) {
+        float lo, hi;
+        upk(x[i], lo, hi);
+        S[2 * i] = k == 0 ? bd * (double)lo : fma(bd, (double)lo, S[2 * i]);
+        S[2 * i + 1] = k == 0 ? bd * (double)hi : fma(bd, (double)hi, S[2 * i + 1]);
+      }
+    }
     if (k == 0) {
 #pragma unroll
       for (int i = 0; i < NP2; ++i) { np[i] = x[i] ^ 0x8000000080000000ull; s1[i] = 0ull; s2[i] = 0ull; }
@@ -349,7 +372,14 @@ __device__ __forceinline__ void finish4(Acc<KT, VEC>& a, const StepArgs& A, floa
   }
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
-    const float g = s1[e] - p[e];                // p holds the negated pivot
+    double g64 = 0.0;
+    float g;
+    if constexpr (Acc<KT, VEC>::WIDE) {
+      g64 = a.S[E0 + e] * A.rB;
+      g = (float)g64;
+    } else {
+      g = s1[e] - p[e];                          // p holds the negated pivot
+    }
     dv[E0 + e] = fmaf(-A.Bf * s1[e], s1[e], s2[e]);
     nv[E0 + e] = g * g;
     a.c = fmaf(g, pv[e], a.c);
@@ -367,6 +397,10 @@ __device__ __forceinline__ void finish4(Acc<KT, VEC>& a, const StepArgs& A, floa
       a.su2 = fmaf(gh, gh, a.su2);
       m[e] = mn;
       vv[e] = vn;
+    } else if constexpr (Acc<KT, VEC>::WIDE) {
+      const double mn = fma(A.beta64, (double)m[e], g64);
+      th[e] = (float)fma(-A.lr64, mn, (double)th[e]);
+      m[e] = (float)mn;
     } else {
       const float mn = fmaf(A.beta, m[e], g);
       th[e] = fmaf(-A.lr, mn, th[e]);
@@ -424,7 +458,7 @@ __device__ __forceinline__ void direct_tile(Acc<KT, Elem<BF16>::VEC>& a, const S
       }
 #pragma unroll
       for (int u = 0; u < U; ++u) {
-        if (k0 + u < KT && k0 + u < A.K) a.add(k0 + u, x[u], A.w[k0 + u], A.bf[k0 + u]);
+        if (k0 + u < KT && k0 + u < A.K) a.add(k0 + u, x[u], A.w[k0 + u], A.bf[k0 + u], A.bd[k0 + u]);
       }
     }
   }
@@ -966,7 +1000,7 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
               if (s * G + u < KT && s * G + u < A.K) {
                 u64 x[VEC / 2];
                 unpack2<BF16>(r[u], x);
-                a.add(s * G + u, x, A.w[s * G + u], A.bf[s * G + u]);
+                a.add(s * G + u, x, A.w[s * G + u], A.bf[s * G + u], A.bd[s * G + u]);
               }
             }
           }

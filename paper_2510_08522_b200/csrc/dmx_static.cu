@@ -16,9 +16,12 @@
 #include <cstring>
 #include <mutex>
 
+#include "dmx_host.h"
 #include "dmx_kernels.cuh"
 
 namespace {
+
+using dmxh::cuda_ok;
 
 constexpr size_t kScratchBytes = DMX_STATIC_SCRATCH_BYTES;
 
@@ -147,8 +150,8 @@ __global__ void __launch_bounds__(NW * 32) static_step_kernel(const __grid_const
   }
 }
 
-// Second level for the static path: one CTA; fp64, fixed order. The derived scalars repeat
-// the formulas of the handle path's finalize kernel.
+// Second level for the static path: one CTA; fp64, fixed order. The derived scalars come from
+// the same device function as the handle path's (dmx::emit_header).
 __global__ void __launch_bounds__(NW * 32) static_finalize_kernel(const __grid_constant__ StaticFinal F) {
   __shared__ double cs[dmx::kMaxK + 2 + 2 * DMX_STATIC_MAX_SEGMENTS];
   __shared__ double s_red[2][NW];
@@ -188,23 +191,7 @@ __global__ void __launch_bounds__(NW * 32) static_finalize_kernel(const __grid_c
     for (int w = 0; w < NW; ++w) { D += s_red[0][w]; A += s_red[1][w]; }
     bool bad = false;
     for (int k = 0; k < K; ++k) { Qw += F.b[k] * cs[k]; bad = bad || !isfinite((float)cs[k]); }
-    const double c = cs[K], pp = cs[K + 1], B = F.B;
-    int flags = 0;
-    double trS = 0.0;
-    if (K >= 2) trS = D / (double)(K - 1); else flags |= DMX_FLAG_SINGLE;
-    const double G2 = A - trS / B;
-    double gns = 0.0;
-    if (G2 > 0.0) gns = trS / G2; else flags |= DMX_FLAG_G2_NONPOS;
-    double cosv = 0.0;
-    if (A > 0.0 && pp > 0.0) cosv = c / sqrt(A * pp); else flags |= DMX_FLAG_COS_UNDEF;
-    const double sig2 = A > 0.0 ? trS / (B * A) : 0.0;
-    const double sig = sqrt(sig2 > 0.0 ? sig2 : 0.0);
-    if (bad || !isfinite((float)A) || !isfinite((float)pp)) flags |= DMX_FLAG_NONFINITE;
-    out[DMX_ST_B_TOTAL] = (float)B; out[DMX_ST_AGG_SQNORM] = (float)A; out[DMX_ST_TR_SIGMA] = (float)trS;
-    out[DMX_ST_G2] = (float)G2; out[DMX_ST_GNS] = (float)gns; out[DMX_ST_COS_PREV] = (float)cosv;
-    out[DMX_ST_DOT_PREV] = (float)c; out[DMX_ST_PREV_SQNORM] = (float)pp; out[DMX_ST_SIGMA2_NORM] = (float)sig2;
-    out[DMX_ST_SIGMA_NORM] = (float)sig; out[DMX_ST_WMEAN_SQNORM] = (float)(Qw / B); out[DMX_ST_FLAGS] = (float)flags;
-    out[12] = out[13] = out[14] = out[15] = 0.f;
+    dmx::emit_header(out, K, F.B, D, A, Qw, cs[K], cs[K + 1], bad, false, 0, 0.0, 0.0, 0.0);
   }
 }
 
@@ -228,17 +215,14 @@ std::mutex g_mu;
 
 int device_scratch(DeviceInfo** out) {
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DMX_ERR_CUDA;
+  if (!cuda_ok(cudaGetDevice(&dev)) || dev < 0 || dev >= kMaxDevices) return DMX_ERR_CUDA;
   std::lock_guard<std::mutex> lock(g_mu);
   DeviceInfo& d = g_dev[dev];
   if (!d.ready) {
     void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_scratch) != cudaSuccess || !p) { (void)cudaGetLastError(); return DMX_ERR_CUDA; }
+    if (!cuda_ok(cudaGetSymbolAddress(&p, g_scratch)) || !p) return DMX_ERR_CUDA;
     int sms = 0;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
-      (void)cudaGetLastError();
-      return DMX_ERR_CUDA;
-    }
+    if (!cuda_ok(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) || sms < 1) return DMX_ERR_CUDA;
     d.scratch = static_cast<unsigned char*>(p);
     d.sms = sms;
     d.ready = true;
@@ -248,11 +232,6 @@ int device_scratch(DeviceInfo** out) {
 }
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
-
-bool ranges_overlap(const void* a, size_t na, const void* b, size_t nb) {
-  const uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
-  return x < y + nb && y < x + na;
-}
 
 }  // namespace
 
@@ -268,29 +247,12 @@ extern "C" int dmx_step_static(int K, int64_t P, const int64_t* seg_offsets, int
   if (seg_offsets[0] != 0 || seg_offsets[S] != P) return DMX_ERR_SEGMENTS;
   for (int s = 0; s < S; ++s)
     if (seg_offsets[s] > seg_offsets[s + 1]) return DMX_ERR_SEGMENTS;
-  const size_t esz = grad_dtype == DMX_BF16 ? 2 : 4;
-  const size_t gbytes = (size_t)P * esz, sbytes = (size_t)P * 4;
-  const size_t obytes = (size_t)(DMX_ST_HDR + K + 2 * S) * 4;
+  const dmxh::StepBuffers sb = {grad_ptrs, batch_sizes, params, momentum, prev_agg, nullptr, out_state,
+                                (size_t)(DMX_ST_HDR + K + 2 * S) * 4, 3u};
   int64_t B = 0;
   int pivot = 0;
-  for (int k = 0; k < K; ++k) {
-    if (!grad_ptrs[k]) return DMX_ERR_ARG;
-    if (batch_sizes[k] < 1) return DMX_ERR_BATCH;
-    B += batch_sizes[k];
-    if (batch_sizes[k] > batch_sizes[pivot]) pivot = k;
-  }
-  for (int k = 0; k < K; ++k)
-    if ((uintptr_t)grad_ptrs[k] & 15) return DMX_ERR_ALIGN;
-  if (((uintptr_t)params & 15) || ((uintptr_t)momentum & 15) || ((uintptr_t)prev_agg & 15) || ((uintptr_t)out_state & 3))
-    return DMX_ERR_ALIGN;
-  const void* st[4] = {params, momentum, prev_agg, out_state};
-  const size_t sn[4] = {sbytes, sbytes, sbytes, obytes};
-  for (int i = 0; i < 4; ++i) {
-    for (int j = i + 1; j < 4; ++j)
-      if (ranges_overlap(st[i], sn[i], st[j], sn[j])) return DMX_ERR_ARG;
-    for (int k = 0; k < K; ++k)
-      if (ranges_overlap(st[i], sn[i], grad_ptrs[k], gbytes)) return DMX_ERR_ARG;
-  }
+  const int rcb = dmxh::check_step_buffers(K, P, grad_dtype, sb, &B, &pivot);
+  if (rcb != DMX_OK) return rcb;
 
   DeviceInfo* dev = nullptr;
   const int rc = device_scratch(&dev);
@@ -313,19 +275,8 @@ extern "C" int dmx_step_static(int K, int64_t P, const int64_t* seg_offsets, int
   std::memset(&A, 0, sizeof(A));
   std::memset(&X, 0, sizeof(X));
   std::memset(&F, 0, sizeof(F));
-  int slot = 0;
-  for (int i = -1; i < K; ++i) {      // the worker with the largest batch first, as in dmx_step
-    const int k = i < 0 ? pivot : i;
-    if (i >= 0 && k == pivot) continue;
-    A.grad[slot] = grad_ptrs[k];
-    A.w[slot] = (float)((double)batch_sizes[k] / (double)B);
-    A.bf[slot] = (float)batch_sizes[k];
-    F.orig[slot] = k;
-    F.b[slot] = (double)batch_sizes[k];
-    ++slot;
-  }
+  dmxh::pack_workers(K, grad_ptrs, batch_sizes, pivot, B, lr, beta, A, F.orig, F.b);   // as in dmx_step
   A.params = params; A.momentum = momentum; A.prev = prev_agg;
-  A.lr = lr; A.beta = beta; A.Bf = (float)B;
   A.K = K; A.S = S; A.P = P;
   X.grid = grid; X.ntiles = ntiles;
   X.seg_off = reinterpret_cast<const int64_t*>(dev->scratch + off_seg);
@@ -337,15 +288,13 @@ extern "C" int dmx_step_static(int K, int64_t P, const int64_t* seg_offsets, int
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   // the segment table travels host -> scratch on the stream (pageable source: the runtime
   // has taken its copy when the call returns)
-  if (cudaMemcpyAsync(dev->scratch + off_seg, seg_offsets, (size_t)(S + 1) * sizeof(int64_t), cudaMemcpyHostToDevice,
-                      stream) != cudaSuccess) {
-    (void)cudaGetLastError();
+  if (!cuda_ok(cudaMemcpyAsync(dev->scratch + off_seg, seg_offsets, (size_t)(S + 1) * sizeof(int64_t),
+                               cudaMemcpyHostToDevice, stream)))
     return DMX_ERR_CUDA;
-  }
   StaticKernel kern = bf16 ? pick_kernel<true>(K) : pick_kernel<false>(K);
   kern<<<grid, NW * 32, 0, stream>>>(A, X);
-  if (cudaGetLastError() != cudaSuccess) return DMX_ERR_CUDA;
+  if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
   static_finalize_kernel<<<1, NW * 32, 0, stream>>>(F);
-  if (cudaGetLastError() != cudaSuccess) return DMX_ERR_CUDA;
+  if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
   return DMX_OK;
 }
