@@ -1,7 +1,7 @@
 /*
  * dmx.h — C ABI of the DYNAMIX data-parallel gradient step on one GPU.
  *
- * The operation (Algorithm 1, the inner "for each worker in parallel" body: each worker
+ * The operation (Algorithm 1, the body of the innermost loop over the workers: each worker
  * computes a gradient g_i at its own batch size x_i and the global model is updated under
  * BSP; Section "State representation", paragraph "Training Statistical Efficiency Metrics":
  * the controller reads gradient statistics, sigma_norm and sigma^2_norm):
@@ -22,6 +22,12 @@
  *     not allocate, does not synchronise and copies nothing host-to-device (worker pointers,
  *     weights and batch sizes travel as kernel arguments).
  *   - A handle may be used from one stream at a time (its scratch is shared by its calls).
+ *   - A handle belongs to the CUDA device that was current in dmx_create: its tables and scratch
+ *     live there. A step issued while another device is current returns DMX_ERR_HANDLE before
+ *     anything is enqueued (make the handle's device current first).
+ *   - Handles are looked up in a table of live handles, never read through the pointer first:
+ *     a call on a destroyed (or never created) handle returns DMX_ERR_HANDLE and touches no
+ *     freed memory. An address reused by a later create names that later handle.
  *   - dmx_step, dmx_step_adam and their _partial forms enqueue two kernel launches and nothing
  *     else, so (with per-kernel timing off) they can be captured in a CUDA graph and replayed:
  *     the kernels leave the handle's scratch ready for the next run.
@@ -49,8 +55,9 @@ enum {
   DMX_ERR_ALIGN = -4,    /* a device pointer is not 16-byte aligned                        */
   DMX_ERR_NOMEM = -5,    /* host or device allocation failed                               */
   DMX_ERR_CUDA = -6,     /* a CUDA runtime call failed (see dmx_last_cuda_error)           */
-  DMX_ERR_HANDLE = -7,   /* handle is NULL, destroyed or corrupt                           */
-  DMX_ERR_LIMIT = -8     /* problem too large for the fixed scratch of dmx_step_static     */
+  DMX_ERR_HANDLE = -7,   /* handle is NULL, destroyed, or belongs to another CUDA device   */
+  DMX_ERR_LIMIT = -8,    /* problem too large for the fixed scratch of dmx_step_static     */
+  DMX_ERR_GUARD = -9     /* dmx_check_guards: a guard word beside the scratch was overwritten */
 };
 
 /* limits */
@@ -90,7 +97,9 @@ enum {
   DMX_FLAG_G2_NONPOS = 2,  /* |G|^2^ <= 0 (or NaN): gns reported as 0                      */
   DMX_FLAG_COS_UNDEF = 4,  /* A == 0 or |a|^2 == 0 (first step): cosine reported as 0      */
   DMX_FLAG_SINGLE = 8,     /* K == 1: no across-worker variance                            */
-  DMX_FLAG_INTERNAL = 16   /* a bounded wait inside the kernel ran out; results invalid    */
+  DMX_FLAG_INTERNAL = 16,  /* a bounded wait inside the kernel ran out; results invalid    */
+  DMX_FLAG_BOUNDS = 32     /* checked build only: an index into the tables or the scratch was
+                              out of range and the access was skipped; results invalid     */
 };
 
 /*
@@ -103,7 +112,12 @@ enum {
  *   S            number of segments, 1..DMX_MAX_SEGMENTS
  *   grad_dtype   DMX_F32 or DMX_BF16 (params, momentum, prev_agg, out_state are fp32)
  *   out          HOST, receives the handle
- * Errors: DMX_ERR_ARG, DMX_ERR_SEGMENTS, DMX_ERR_NOMEM, DMX_ERR_CUDA. Synchronous.
+ * Errors: DMX_ERR_ARG, DMX_ERR_SEGMENTS, DMX_ERR_NOMEM, DMX_ERR_CUDA. Synchronous. On any error
+ * everything allocated so far is released and *out is NULL.
+ * For tests of that clean-up: with the environment variable DMX_TEST_FAIL_ALLOC=n the n-th
+ * allocation of a create call (counted from 1, the handle structure first, then the device
+ * buffers) is refused on the host as if memory had run out; no device call is made for it.
+ * dmx_agg_create honours the same variable.
  */
 int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dtype,
                dmx_handle** out);
@@ -137,8 +151,8 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
 
 /*
  * dmx_step_adam — the same pass with the Adam update in place of SGD with momentum (the paper
- * evaluates both optimizers, Section "Workloads and Datasets", and reads sigma_norm and
- * sigma^2_norm "for adaptive optimizers", Section "State representation"). With g the
+ * evaluates both optimizers, Section "Workloads and Datasets", and its state vector carries
+ * sigma_norm and sigma^2_norm when the optimizer is adaptive, Section "State representation"). With g the
  * aggregate (Kingma & Ba 2015, Algorithm 1, bias-corrected form):
  *   m' = beta1 m + (1-beta1) g          v' = beta2 v + (1-beta2) g^2
  *   mhat = m' / (1-beta1^t)             vhat = v' / (1-beta2^t)
@@ -185,8 +199,9 @@ enum { DMX_ST_ADAM_GHAT_MEAN = 12, DMX_ST_ADAM_GHAT_VAR = 13, DMX_ST_ADAM_GHAT_S
  *                       but instead of out_state they write `partials` (DEVICE, dmx_partials_len
  *                       doubles, 8-byte aligned): q_k [K] in the caller's worker order, <g,a>, |a|^2,
  *                       Adam's sum and sum of squares of ghat (0 for SGD), Vraw_s [S] (before the
- *                       division by K-1), N_s [S], and a word that is non-zero if a bounded wait
- *                       inside the kernel ran out.
+ *                       division by K-1), N_s [S], and an error word (1 if a bounded wait inside
+ *                       the kernel ran out, plus 65536 if the checked build found an index out
+ *                       of range; added over the shards like the rest).
  *   dmx_finalize_partials
  *                       batch_sizes: HOST, K ints; partials: DEVICE, the entry-wise sum over all
  *                       shards; P_total: the whole problem's parameter count (Adam's mean); writes
@@ -235,8 +250,32 @@ int dmx_step_host(dmx_handle* h, const void* const* host_grad_ptrs, void* const*
 int dmx_set_profiling(dmx_handle* h, int on);
 int dmx_get_profile(dmx_handle* h, float* fused_ms, float* finalize_ms);
 
-/* Number of kernels one dmx_step launches (2: fused pass, finalize). */
+/* Number of kernels one dmx_step launches: 1 when the problem's reduction scratch is small
+ * enough for the fused pass to do the second level itself (a few hundred chunks, at most 512
+ * segments), else 2 (fused pass, finalize). */
 int dmx_launches_per_step(const dmx_handle* h);
+
+/*
+ * Checks of the library's own machinery (the paper has no counterpart; robustness is one of its
+ * stated requirements, and these are how this library shows it without ever faulting a GPU).
+ *
+ * dmx_check_guards — every scratch array a handle's kernels write lies between two guard regions
+ *   filled with a fixed word by dmx_create. This reads them back (synchronous copies; call it when
+ *   no step of the handle is running) and returns DMX_OK, or DMX_ERR_GUARD if a word has changed,
+ *   i.e. some kernel wrote just outside its array.
+ *
+ * dmx_selftest_wait — every wait inside the fused pass is bounded: after a fixed number of polls
+ *   it gives up, raises the handle's error word and the CTA drains; the step's state vector then
+ *   carries DMX_FLAG_INTERNAL and the word is cleared for the next step. This launches one warp
+ *   that waits, with a budget of `polls` (1..2^24) polls, on a barrier that nothing will ever
+ *   complete (no copy in flight, nobody to arrive): the wait must run out. *timed_out (HOST)
+ *   receives 1 if it did; *waited_ms (HOST) the time the warp spent waiting, by the GPU's timer.
+ *   The handle's error word is raised exactly as by a failed wait in a step: the next step of the
+ *   handle reports DMX_FLAG_INTERNAL (its other outputs are valid) and clears it. Synchronous.
+ *   Errors: DMX_ERR_HANDLE, DMX_ERR_ARG, DMX_ERR_NOMEM, DMX_ERR_CUDA.
+ */
+int dmx_check_guards(dmx_handle* h);
+int dmx_selftest_wait(dmx_handle* h, uint32_t polls, int* timed_out, double* waited_ms, void* cuda_stream);
 
 /*
  * dmx_plan_chunks — the work list dmx_create builds for the fused pass (host only: no CUDA call,
@@ -251,7 +290,8 @@ int dmx_launches_per_step(const dmx_handle* h);
  *                   number of CTAs the kernel is launched with
  *   first_tile, num_tiles, group_stride   HOST, capacity entries each (may be NULL with capacity 0)
  * Returns the number of chunks (the arrays are filled only if capacity is at least that), or
- * DMX_ERR_ARG.
+ * DMX_ERR_ARG. The tuning variables dmx_create reads (DMX_TILE_GROUP, DMX_CHUNK_TILES,
+ * DMX_MIN_CHUNK_KB) apply here too.
  */
 int dmx_plan_chunks(int64_t P, int K, int grad_dtype, int tile_elems, int resident_ctas,
                     int32_t* first_tile, int32_t* num_tiles, int32_t* group_stride, int capacity,
@@ -343,8 +383,13 @@ int dmx_ctl_decide(int K, int M, int H, int state_len, const float* window, cons
  * DMX_STATIC_SCRATCH_BYTES inside the library's device image: every GPU on which the library
  * is loaded holds that array until the process exits.
  *
- *   K, P, seg_offsets, S, grad_dtype   as dmx_create (seg_offsets is HOST memory, read during
- *                                      the call), but S <= DMX_STATIC_MAX_SEGMENTS
+ *   K, P, seg_offsets, S, grad_dtype   as dmx_create, but S <= DMX_STATIC_MAX_SEGMENTS.
+ *                                      seg_offsets is HOST memory. It is validated during the call
+ *                                      and copied to the device by an asynchronous copy on the
+ *                                      stream: from pageable memory the runtime has taken its copy
+ *                                      when the call returns; from pinned memory the table must
+ *                                      stay unchanged until the stream has passed the call (and
+ *                                      for as long as a captured copy of the call may be replayed)
  *   grad_ptrs ... cuda_stream          as dmx_step
  *
  * It calls no cudaMalloc, cudaFree or other allocating routine; the caller still provides
@@ -368,8 +413,8 @@ int dmx_step_static(int K, int64_t P, const int64_t* seg_offsets, int S, int gra
                     float* momentum, float lr, float beta, float* prev_agg, float* out_state,
                     void* cuda_stream);
 
-/* Frees the tables and the scratch. NULL is accepted. The caller makes sure no step of
- * this handle is still running. */
+/* Frees the tables and the scratch. NULL is accepted; a handle that is not live (destroyed
+ * already) gives DMX_ERR_HANDLE. The caller makes sure no step of this handle is still running. */
 int dmx_destroy(dmx_handle* h);
 
 /* Static, NUL-terminated description of a return code. */

@@ -7,8 +7,8 @@
 //
 // What it computes is the plain definition of the step, one parameter at a time, in
 // fp64, in the order and notation of the method:
-//   Algorithm 1, worker loop ("compute gradient g_i and update global model"): the K
-//     workers' gradients x_k (each a mean over b_k samples) are combined into the mean
+//   Algorithm 1, worker loop (each worker computes its gradient at its own batch size and the
+//     global model is updated): the K workers' gradients x_k (each a mean over b_k samples) are combined into the mean
 //     over all B = sum b_k samples, g_j = (sum_k b_k x_kj) / B, and the global model takes
 //     one SGD-momentum step m <- beta m + g, theta <- theta - lr m (Section "Workloads
 //     and Datasets" names SGD; the momentum form is the usual undampened one), or one Adam

@@ -12,18 +12,18 @@ from . import build as _build
 
 F32, BF16 = 0, 1
 OK = 0
-ERR_ARG, ERR_SEGMENTS, ERR_BATCH, ERR_ALIGN, ERR_NOMEM, ERR_CUDA, ERR_HANDLE, ERR_LIMIT = -1, -2, -3, -4, -5, -6, -7, -8
+ERR_ARG, ERR_SEGMENTS, ERR_BATCH, ERR_ALIGN, ERR_NOMEM, ERR_CUDA, ERR_HANDLE, ERR_LIMIT, ERR_GUARD = -1, -2, -3, -4, -5, -6, -7, -8, -9
 STATIC_MAX_SEGMENTS, STATIC_SCRATCH_BYTES = 512, 1 << 20
 ST_B_TOTAL, ST_AGG_SQNORM, ST_TR_SIGMA, ST_G2, ST_GNS, ST_COS_PREV, ST_DOT_PREV, ST_PREV_SQNORM = range(8)
 ST_SIGMA2_NORM, ST_SIGMA_NORM, ST_WMEAN_SQNORM, ST_FLAGS = 8, 9, 10, 11
 ST_HDR = 16
-FLAG_NONFINITE, FLAG_G2_NONPOS, FLAG_COS_UNDEF, FLAG_SINGLE, FLAG_INTERNAL = 1, 2, 4, 8, 16
+FLAG_NONFINITE, FLAG_G2_NONPOS, FLAG_COS_UNDEF, FLAG_SINGLE, FLAG_INTERNAL, FLAG_BOUNDS = 1, 2, 4, 8, 16, 32
 
 EXPORTS = ("dmx_create", "dmx_state_len", "dmx_step", "dmx_step_adam", "dmx_step_host", "dmx_step_static", "dmx_set_profiling", "dmx_get_profile",
            "dmx_launches_per_step", "dmx_destroy", "dmx_strerror", "dmx_last_cuda_error", "dmx_agg_create",
            "dmx_agg_push", "dmx_agg_destroy", "dmx_ctl_num_features", "dmx_ctl_num_weights", "dmx_ctl_decide", "dmx_plan_chunks",
            "dmx_shard_range", "dmx_shard_segments", "dmx_partials_len", "dmx_step_partial", "dmx_step_adam_partial",
-           "dmx_finalize_partials")
+           "dmx_finalize_partials", "dmx_check_guards", "dmx_selftest_wait")
 CTL_ACTIONS = (-100, -25, 0, 25, 100)
 
 _lib = None
@@ -36,10 +36,13 @@ class DmxError(RuntimeError):
 
 
 def lib():
-    """Load lib/libdmx.so (built in-tree by `python -m paper_2510_08522_b200.build`)."""
+    """Load lib/libdmx.so (built in-tree by `python -m paper_2510_08522_b200.build`). With the
+    environment variable DMX_CHECKED_BUILD=1 the checked build lib/libdmx_checked.so is loaded
+    instead (`python -m paper_2510_08522_b200.build --checked`): same ABI, every table and scratch
+    index range-tested on the device."""
     global _lib
     if _lib is None:
-        path = _build.lib_path("libdmx.so")
+        path = _build.lib_path("libdmx_checked.so" if os.environ.get("DMX_CHECKED_BUILD") == "1" else "libdmx.so")
         if not os.path.exists(path):
             raise RuntimeError("CUDA library %s is not built; run `python -m paper_2510_08522_b200.build`" % path)
         L = ctypes.CDLL(path)
@@ -89,6 +92,10 @@ def lib():
         L.dmx_get_profile.restype = i32
         L.dmx_launches_per_step.argtypes = [vp]
         L.dmx_launches_per_step.restype = i32
+        L.dmx_check_guards.argtypes = [vp]
+        L.dmx_check_guards.restype = i32
+        L.dmx_selftest_wait.argtypes = [vp, ctypes.c_uint32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_double), vp]
+        L.dmx_selftest_wait.restype = i32
         L.dmx_destroy.argtypes = [vp]
         L.dmx_destroy.restype = i32
         L.dmx_strerror.argtypes = [i32]
@@ -304,6 +311,17 @@ def dmx_launches_per_step(h) -> int:
     return lib().dmx_launches_per_step(h)
 
 
+def dmx_check_guards(h) -> int:
+    return lib().dmx_check_guards(h)
+
+
+def dmx_selftest_wait(h, polls, stream=0):
+    """-> (code, timed_out, waited_ms): one warp waits `polls` polls on a barrier nothing completes."""
+    t, ms = ctypes.c_int(0), ctypes.c_double(0.0)
+    rc = lib().dmx_selftest_wait(h, int(polls), ctypes.byref(t), ctypes.byref(ms), int(stream) if stream else None)
+    return rc, t.value, ms.value
+
+
 def dmx_destroy(h) -> int:
     return lib().dmx_destroy(h)
 
@@ -398,6 +416,11 @@ class Dmx:
     @property
     def launches_per_step(self):
         return dmx_launches_per_step(self._h)
+
+    def check_guards(self):
+        rc = dmx_check_guards(self._h)
+        if rc != OK:
+            raise DmxError(rc, "dmx_check_guards")
 
     def close(self):
         if getattr(self, "_h", None):

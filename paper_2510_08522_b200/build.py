@@ -1,7 +1,10 @@
-"""In-tree build of the two shared objects (nvcc, sm_100a only):
-    lib/libdmx.so      the gradient-step library (C ABI of include/dmx.h)
-    lib/libdmx_gen.so  the synthetic-input fill kernels
-Run as `python -m paper_2510_08522_b200.build [--force] [--verbose]`.
+"""In-tree build of the shared objects (nvcc, sm_100a only):
+    lib/libdmx.so          the gradient-step library (C ABI of include/dmx.h)
+    lib/libdmx_gen.so      the synthetic-input fill kernels
+    lib/libdmx_checked.so  (with --checked) the gradient-step library compiled with -DDMX_DEBUG:
+                           every index into the tables and the scratch is range-tested on the
+                           device; a violation sets DMX_FLAG_BOUNDS in the state vector, never a trap
+Run as `python -m paper_2510_08522_b200.build [--force] [--verbose] [--checked]`.
 """
 from __future__ import annotations
 
@@ -35,15 +38,22 @@ def lib_path(name: str) -> str:
     return os.path.join(LIBDIR, name)
 
 
-def build(force: bool = False, verbose: bool = False) -> None:
+CHECKED = {"libdmx_checked.so": TARGETS["libdmx.so"]}
+
+
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> None:
     os.makedirs(LIBDIR, exist_ok=True)
-    for name, (srcs, deps) in TARGETS.items():
+    targets = dict(TARGETS)
+    if checked:
+        targets.update(CHECKED)
+    for name, (srcs, deps) in targets.items():
         out = lib_path(name)
         srcs_abs = [os.path.join(CSRC, s) for s in srcs]
         deps_abs = srcs_abs + [d if os.path.isabs(d) else os.path.join(CSRC, d) for d in deps]
         if not force and os.path.exists(out) and all(os.path.getmtime(out) >= os.path.getmtime(d) for d in deps_abs):
             continue
-        cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + srcs_abs + ["-o", out + ".tmp"]
+        cmd = ([_nvcc()] + NVCC_FLAGS + (["-DDMX_DEBUG"] if name in CHECKED else []) +
+               (["-Xptxas", "-v"] if verbose else []) + srcs_abs + ["-o", out + ".tmp"])
         if verbose:
             print(" ".join(cmd), flush=True)
         subprocess.check_call(cmd)
@@ -51,4 +61,4 @@ def build(force: bool = False, verbose: bool = False) -> None:
 
 
 if __name__ == "__main__":
-    build(force="--force" in sys.argv, verbose="--verbose" in sys.argv)
+    build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, checked="--checked" in sys.argv)

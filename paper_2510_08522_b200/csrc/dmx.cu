@@ -6,7 +6,9 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
+#include <unordered_map>
 #include <vector>
 
 #include "dmx_host.h"
@@ -14,6 +16,9 @@
 
 namespace {
 thread_local int g_last_cuda = 0;
+thread_local int g_alloc_count = 0, g_alloc_fail = 0;
+std::mutex g_live_mu;
+std::unordered_map<const void*, int> g_live;
 }
 
 namespace dmxh {
@@ -76,6 +81,43 @@ void pack_workers(int K, const void* const* grad_ptrs, const int32_t* batch_size
   A.rB = 1.0 / (double)B; A.lr64 = (double)lr; A.beta64 = (double)beta;
 }
 
+void live_add(const void* p, int kind) {
+  std::lock_guard<std::mutex> lock(g_live_mu);
+  g_live[p] = kind;
+}
+
+bool live_has(const void* p, int kind) {
+  if (!p) return false;
+  std::lock_guard<std::mutex> lock(g_live_mu);
+  const auto it = g_live.find(p);
+  return it != g_live.end() && it->second == kind;
+}
+
+bool live_remove(const void* p, int kind) {
+  std::lock_guard<std::mutex> lock(g_live_mu);
+  const auto it = g_live.find(p);
+  if (it == g_live.end() || it->second != kind) return false;
+  g_live.erase(it);
+  return true;
+}
+
+void alloc_begin() {
+  g_alloc_count = 0;
+  const char* v = std::getenv("DMX_TEST_FAIL_ALLOC");
+  g_alloc_fail = (v && *v) ? std::atoi(v) : 0;
+}
+
+bool alloc_host_ok() { return ++g_alloc_count != g_alloc_fail; }
+
+bool dev_alloc(void** p, size_t bytes) {
+  *p = nullptr;
+  if (++g_alloc_count == g_alloc_fail) {
+    g_last_cuda = (int)cudaErrorMemoryAllocation;
+    return false;
+  }
+  return cuda_ok(cudaMalloc(p, bytes));
+}
+
 int check_current_device(int device) {
   int cur = -1;
   if (!cuda_ok(cudaGetDevice(&cur))) return DMX_ERR_CUDA;
@@ -88,9 +130,9 @@ namespace {
 
 using dmxh::cuda_ok;
 
-constexpr uint64_t kMagic = 0x444d585f48414e44ull;  // "DMX_HAND"
+bool live(const dmx_handle* h) { return dmxh::live_has(h, dmxh::kStepHandle); }
 
-typedef void (*StepKernel)(const dmx::StepArgs);
+typedef void (*StepKernel)(const dmx::StepArgs, const dmx::FinalArgs);
 
 struct Plan {
   StepKernel kernel = nullptr;       // SGD-momentum update
@@ -111,29 +153,33 @@ template <typename T>
 bool upload(const std::vector<T>& v, T** dptr) {
   *dptr = nullptr;
   if (v.empty()) return true;
-  if (!cuda_ok(cudaMalloc((void**)dptr, v.size() * sizeof(T)))) return false;
+  if (!dmxh::dev_alloc((void**)dptr, v.size() * sizeof(T))) return false;
   return cuda_ok(cudaMemcpy(*dptr, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice));
 }
 
 }  // namespace
 
 struct dmx_handle {
-  uint64_t magic = kMagic;
   int K = 0, S = 0, dtype = 0, device = 0;
   int64_t P = 0;
   Plan plan;
   int nchunks = 0, nslots = 0, tile_group = 1;
+  int64_t ntiles = 0;
+  bool fold = false;     // the fused pass runs the second level itself (one launch per step)
   // device tables
   int64_t* seg_off = nullptr;
   int32_t *tile_seg = nullptr, *chunk_stride = nullptr, *chunk_tile0 = nullptr, *chunk_ntiles = nullptr;
-  int32_t *chunk_slot0 = nullptr, *seg_slots = nullptr, *unit_lo = nullptr, *unit_hi = nullptr, *seg_unit_ptr = nullptr;
+  int32_t *chunk_slot0 = nullptr, *slot_dest = nullptr, *seg_ptr = nullptr, *unit_lo = nullptr, *unit_hi = nullptr,
+          *seg_unit_ptr = nullptr;
   double2* segpart = nullptr;
   int nunits = 0;
-  // device scratch
+  // device scratch; each array sits between two guard regions (see alloc_guarded)
   float* rows = nullptr;
   float2* slots = nullptr;
   double* colsum = nullptr;
   unsigned* flags = nullptr;  // [0] ticket, [1] err, [2] the fused pass's chunk counter
+  struct Guarded { unsigned char* raw; size_t bytes; };
+  std::vector<Guarded> guarded;
   // optional per-kernel timing
   bool profiling = false, profiled = false;
   cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
@@ -282,16 +328,39 @@ void plan_chunks(int64_t P, int K, int grad_dtype, int tile, int64_t sm_ctas, in
   }
 }
 
+// Scratch that kernels write is allocated between two guard regions of kGuardBytes filled with a
+// fixed word; dmx_check_guards reads them back. A write that strays just outside its array (the
+// kind of bug no result check would notice if it landed in a neighbouring allocation) shows
+// there. The array itself starts 256-byte aligned.
+constexpr size_t kGuardBytes = 256;
+constexpr uint32_t kGuardWord = 0x5afe6a4du;
+
+template <typename T>
+bool alloc_guarded(dmx_handle* h, T** p, size_t bytes) {
+  *p = nullptr;
+  const size_t body = (bytes + 255) & ~(size_t)255;
+  void* raw = nullptr;
+  if (!dmxh::dev_alloc(&raw, body + 2 * kGuardBytes)) return false;
+  h->guarded.push_back({static_cast<unsigned char*>(raw), body});
+  uint32_t pat[kGuardBytes / 4];
+  for (uint32_t& w : pat) w = kGuardWord;
+  unsigned char* base = static_cast<unsigned char*>(raw);
+  if (!cuda_ok(cudaMemcpy(base, pat, kGuardBytes, cudaMemcpyHostToDevice)) ||
+      !cuda_ok(cudaMemcpy(base + kGuardBytes + body, pat, kGuardBytes, cudaMemcpyHostToDevice)))
+    return false;
+  *p = reinterpret_cast<T*>(base + kGuardBytes);
+  return true;
+}
+
 void free_handle(dmx_handle* h) {
   if (!h) return;
   cudaFree(h->seg_off); cudaFree(h->tile_seg); cudaFree(h->chunk_stride); cudaFree(h->chunk_tile0);
-  cudaFree(h->chunk_ntiles); cudaFree(h->chunk_slot0); cudaFree(h->seg_slots); cudaFree(h->unit_lo);
-  cudaFree(h->unit_hi); cudaFree(h->seg_unit_ptr); cudaFree(h->segpart);
-  cudaFree(h->rows); cudaFree(h->slots); cudaFree(h->colsum); cudaFree(h->flags);
+  cudaFree(h->chunk_ntiles); cudaFree(h->chunk_slot0); cudaFree(h->slot_dest); cudaFree(h->seg_ptr); cudaFree(h->unit_lo);
+  cudaFree(h->unit_hi); cudaFree(h->seg_unit_ptr);
+  for (const dmx_handle::Guarded& g : h->guarded) cudaFree(g.raw);
   for (int i = 0; i < 3; ++i)
     if (h->ev[i]) cudaEventDestroy(h->ev[i]);
   (void)cudaGetLastError();
-  h->magic = 0;
   delete h;
 }
 
@@ -309,7 +378,8 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   for (int s = 0; s < S; ++s)
     if (seg_offsets[s] > seg_offsets[s + 1]) return DMX_ERR_SEGMENTS;
 
-  dmx_handle* h = new (std::nothrow) dmx_handle;
+  dmxh::alloc_begin();
+  dmx_handle* h = dmxh::alloc_host_ok() ? new (std::nothrow) dmx_handle : nullptr;
   if (!h) return DMX_ERR_NOMEM;
   h->K = K; h->P = P; h->S = S; h->dtype = grad_dtype;
   cudaDeviceProp prop;
@@ -368,8 +438,11 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   for (int c = 0; c < nchunks; ++c) {
     chunk_slot0[c] = (int32_t)slot_seg.size();
     int cur = -1;
-    for (int i = 0; i < chunk_ntiles[c]; ++i) {
-      const int64_t t = chunk_tile0[c] + (int64_t)(i / R) * chunk_stride[c] + i % R;
+    const int ntc = chunk_ntiles[c];
+    const auto tile_at = [&](int i) { return chunk_tile0[c] + (int64_t)(i / R) * chunk_stride[c] + i % R; };
+    const bool ragged_last = P % plan.tile != 0 && tile_at(ntc - 1) == ntiles - 1;
+    for (int ii = 0; ii < ntc; ++ii) {
+      const int64_t t = tile_at(dmx::chunk_order(ii, ntc, ragged_last));
       const int64_t j1 = std::min<int64_t>((t + 1) * plan.tile, P);
       const int s0 = tile_seg[(size_t)t] & (dmx::kTileBoundaryBit - 1);
       if (s0 != cur) {
@@ -383,13 +456,14 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
     if (cur >= 0) slot_seg.push_back(cur);
     if (slot_seg.size() > ((size_t)1 << 30)) { free_handle(h); return DMX_ERR_NOMEM; }
   }
+  // the slots are stored grouped by segment (each group in entry order): entry i goes to slot_dest[i]
   const int64_t nslots = (int64_t)slot_seg.size();
-  std::vector<int32_t> seg_ptr(S + 1, 0), seg_slots((size_t)nslots);
+  std::vector<int32_t> seg_ptr(S + 1, 0), slot_dest((size_t)nslots);
   for (int64_t i = 0; i < nslots; ++i) ++seg_ptr[slot_seg[(size_t)i] + 1];
   for (int s = 0; s < S; ++s) seg_ptr[s + 1] += seg_ptr[s];
   {
     std::vector<int32_t> fill(seg_ptr.begin(), seg_ptr.end() - 1);
-    for (int64_t i = 0; i < nslots; ++i) seg_slots[(size_t)fill[slot_seg[(size_t)i]]++] = (int32_t)i;
+    for (int64_t i = 0; i < nslots; ++i) slot_dest[(size_t)i] = fill[slot_seg[(size_t)i]]++;
   }
   // finalize units: runs of at most kFinalPart slots of one segment
   std::vector<int32_t> unit_lo, unit_hi, seg_unit_ptr(S + 1, 0);
@@ -402,17 +476,23 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   }
   seg_unit_ptr[S] = (int32_t)unit_lo.size();
   h->nchunks = nchunks; h->nslots = (int)nslots; h->nunits = (int)unit_lo.size();
+  h->ntiles = ntiles;
+  // Small scratch: the fused pass does the second level itself (one launch per step). DMX_FOLD=0
+  // keeps the separate finalize kernel (a tuning and cross-check knob).
+  h->fold = !direct && env_int("DMX_FOLD", 1) != 0 && (int64_t)(K + 4) * nchunks <= dmx::kFoldMaxRowFloats &&
+            nslots <= dmx::kFoldMaxSlots && S <= dmx::kFoldMaxSegments;
 
   std::vector<int64_t> seg(seg_offsets, seg_offsets + S + 1);
   bool ok = upload(seg, &h->seg_off) && upload(tile_seg, &h->tile_seg) && upload(chunk_stride, &h->chunk_stride) &&
             upload(chunk_tile0, &h->chunk_tile0) && upload(chunk_ntiles, &h->chunk_ntiles) &&
-            upload(chunk_slot0, &h->chunk_slot0) && upload(seg_slots, &h->seg_slots) && upload(unit_lo, &h->unit_lo) &&
+            upload(chunk_slot0, &h->chunk_slot0) && upload(slot_dest, &h->slot_dest) && upload(seg_ptr, &h->seg_ptr) &&
+            upload(unit_lo, &h->unit_lo) &&
             upload(unit_hi, &h->unit_hi) && upload(seg_unit_ptr, &h->seg_unit_ptr);
-  ok = ok && cuda_ok(cudaMalloc((void**)&h->segpart, (size_t)std::max(h->nunits, 1) * sizeof(double2)));
-  ok = ok && cuda_ok(cudaMalloc((void**)&h->rows, (size_t)nchunks * (K + 4) * sizeof(float)));
-  ok = ok && cuda_ok(cudaMalloc((void**)&h->slots, (size_t)std::max<int64_t>(nslots, 1) * sizeof(float2)));
-  ok = ok && cuda_ok(cudaMalloc((void**)&h->colsum, (size_t)(K + 4) * sizeof(double)));
-  ok = ok && cuda_ok(cudaMalloc((void**)&h->flags, 4 * sizeof(unsigned)));
+  ok = ok && alloc_guarded(h, &h->segpart, (size_t)std::max(h->nunits, 1) * sizeof(double2));
+  ok = ok && alloc_guarded(h, &h->rows, (size_t)nchunks * (K + 4) * sizeof(float));
+  ok = ok && alloc_guarded(h, &h->slots, (size_t)std::max<int64_t>(nslots, 1) * sizeof(float2));
+  ok = ok && alloc_guarded(h, &h->colsum, (size_t)(K + 4) * sizeof(double));
+  ok = ok && alloc_guarded(h, &h->flags, 4 * sizeof(unsigned));
   ok = ok && cuda_ok(cudaMemset(h->flags, 0, 4 * sizeof(unsigned)));
   ok = ok && cuda_ok(cudaDeviceSynchronize());
   if (!ok) {
@@ -420,12 +500,13 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
     free_handle(h);
     return nomem ? DMX_ERR_NOMEM : DMX_ERR_CUDA;
   }
+  dmxh::live_add(h, dmxh::kStepHandle);
   *out = h;
   return DMX_OK;
 }
 
 int dmx_state_len(const dmx_handle* h) {
-  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
+  if (!live(h)) return DMX_ERR_HANDLE;
   return DMX_ST_HDR + h->K + 2 * h->S;
 }
 
@@ -440,7 +521,7 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
               float* momentum, float lr, float beta, float* prev_agg, float* out_state, void* cuda_stream,
               const AdamParams* ap, double* partials = nullptr) {
   // `partials` (a parameter shard of a larger problem): the raw sums go there and out_state is not written
-  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
+  if (!live(h)) return DMX_ERR_HANDLE;
   if (!out_state && !partials) return DMX_ERR_ARG;
   if (ap && (!ap->second || ap->t < 1 || !(beta >= 0.f && beta < 1.f) || !(ap->beta2 >= 0.f && ap->beta2 < 1.f) ||
              !(ap->eps >= 0.f)))
@@ -479,12 +560,13 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
   // which also makes a step that was captured in a CUDA graph replayable
   A.next_chunk = h->flags + 2;
   A.seg_off = h->seg_off; A.tile_seg = h->tile_seg; A.chunk_stride = h->chunk_stride; A.chunk_tile0 = h->chunk_tile0;
-  A.chunk_ntiles = h->chunk_ntiles; A.chunk_slot0 = h->chunk_slot0;
+  A.chunk_ntiles = h->chunk_ntiles; A.chunk_slot0 = h->chunk_slot0; A.slot_dest = h->slot_dest;
   A.rows = h->rows; A.slots = h->slots; A.err = h->flags + 1;
+  A.ntiles = (int)h->ntiles; A.nslots = h->nslots;
 
   F.K = K; F.S = h->S; F.nchunks = h->nchunks; F.B = (double)B;
   F.adam = ap ? 1 : 0; F.P = (double)h->P;
-  F.rows = h->rows; F.slots = h->slots; F.seg_slots = h->seg_slots; F.nunits = h->nunits;
+  F.rows = h->rows; F.slots = h->slots; F.seg_ptr = h->seg_ptr; F.nslots = h->nslots; F.nunits = h->nunits;
   F.unit_lo = h->unit_lo; F.unit_hi = h->unit_hi; F.seg_unit_ptr = h->seg_unit_ptr; F.segpart = h->segpart;
   F.colsum = h->colsum; F.ticket = h->flags; F.err = h->flags + 1; F.next_chunk = h->flags + 2;
   F.out_state = out_state;
@@ -493,10 +575,19 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const bool prof = h->profiling;
   if (prof && !cuda_ok(cudaEventRecord(h->ev[0], stream))) return DMX_ERR_CUDA;
-  if (ap) h->plan.kernel_adam<<<h->plan.grid, h->plan.threads, h->plan.smem_adam, stream>>>(A);
-  else h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A);
+  A.fold = h->fold ? 1 : 0;
+  if (ap) h->plan.kernel_adam<<<h->plan.grid, h->plan.threads, h->plan.smem_adam, stream>>>(A, F);
+  else h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A, F);
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
   if (prof && !cuda_ok(cudaEventRecord(h->ev[1], stream))) return DMX_ERR_CUDA;
+  if (h->fold) {
+    // the fused pass has done the second level itself: nothing more to launch
+    if (prof) {
+      if (!cuda_ok(cudaEventRecord(h->ev[2], stream))) return DMX_ERR_CUDA;
+      h->profiled = true;
+    }
+    return DMX_OK;
+  }
   // one block per chunk-row column, one warp per segment unit. Launched as a programmatic
   // dependent of the fused pass: its blocks may become resident while that kernel drains and
   // wait (griddepcontrol.wait) for its completion, which hides the launch latency between the
@@ -539,7 +630,7 @@ int dmx_step_adam(dmx_handle* h, const void* const* grad_ptrs, const int32_t* ba
 }
 
 int dmx_partials_len(const dmx_handle* h) {
-  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
+  if (!live(h)) return DMX_ERR_HANDLE;
   return h->K + 5 + 2 * h->S;
 }
 
@@ -603,8 +694,9 @@ int dmx_shard_segments(const int64_t* seg_offsets, int S, int64_t lo, int64_t hi
 int dmx_step_host(dmx_handle* h, const void* const* host_grad_ptrs, void* const* staging_ptrs,
                   const int32_t* batch_sizes, float* params, float* momentum, float lr, float beta,
                   float* prev_agg, float* out_state_dev, float* out_state_host, void* cuda_stream) {
-  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
+  if (!live(h)) return DMX_ERR_HANDLE;
   if (!host_grad_ptrs || !staging_ptrs || !out_state_host || !out_state_dev) return DMX_ERR_ARG;
+  if (const int rcd = dmxh::check_current_device(h->device); rcd != DMX_OK) return rcd;
   const size_t gbytes = (size_t)h->P * (h->dtype == DMX_BF16 ? 2 : 4);
   for (int k = 0; k < h->K; ++k) {
     if (!host_grad_ptrs[k] || !staging_ptrs[k]) return DMX_ERR_ARG;
@@ -624,7 +716,7 @@ int dmx_step_host(dmx_handle* h, const void* const* host_grad_ptrs, void* const*
 }
 
 int dmx_set_profiling(dmx_handle* h, int on) {
-  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
+  if (!live(h)) return DMX_ERR_HANDLE;
   if (on) {
     for (int i = 0; i < 3; ++i)
       if (!h->ev[i] && !cuda_ok(cudaEventCreate(&h->ev[i]))) return DMX_ERR_CUDA;
@@ -635,7 +727,7 @@ int dmx_set_profiling(dmx_handle* h, int on) {
 }
 
 int dmx_get_profile(dmx_handle* h, float* fused_ms, float* finalize_ms) {
-  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
+  if (!live(h)) return DMX_ERR_HANDLE;
   if (!fused_ms || !finalize_ms || !h->profiling || !h->profiled) return DMX_ERR_ARG;
   if (!cuda_ok(cudaEventSynchronize(h->ev[2]))) return DMX_ERR_CUDA;
   if (!cuda_ok(cudaEventElapsedTime(fused_ms, h->ev[0], h->ev[1]))) return DMX_ERR_CUDA;
@@ -649,7 +741,8 @@ int dmx_plan_chunks(int64_t P, int K, int grad_dtype, int tile_elems, int reside
       (grad_dtype != DMX_F32 && grad_dtype != DMX_BF16) || capacity < 0)
     return DMX_ERR_ARG;
   ChunkPlan cp;
-  plan_chunks(P, K, grad_dtype, tile_elems, resident_ctas, 0, 0, 0, cp);
+  plan_chunks(P, K, grad_dtype, tile_elems, resident_ctas, env_int("DMX_TILE_GROUP", 0), env_int("DMX_CHUNK_TILES", 0),
+              env_int("DMX_MIN_CHUNK_KB", 0), cp);
   if (group_tiles) *group_tiles = cp.R;
   if (grid) *grid = cp.grid;
   const int n = (int)cp.tile0.size();
@@ -662,13 +755,46 @@ int dmx_plan_chunks(int64_t P, int K, int grad_dtype, int tile_elems, int reside
 }
 
 int dmx_launches_per_step(const dmx_handle* h) {
-  if (!h || h->magic != kMagic) return DMX_ERR_HANDLE;
-  return 2;
+  if (!live(h)) return DMX_ERR_HANDLE;
+  return h->fold ? 1 : 2;
+}
+
+int dmx_check_guards(dmx_handle* h) {
+  if (!live(h)) return DMX_ERR_HANDLE;
+  if (const int rc = dmxh::check_current_device(h->device); rc != DMX_OK) return rc;
+  uint32_t got[2 * kGuardBytes / 4];
+  for (const dmx_handle::Guarded& g : h->guarded) {
+    if (!cuda_ok(cudaMemcpy(got, g.raw, kGuardBytes, cudaMemcpyDeviceToHost)) ||
+        !cuda_ok(cudaMemcpy(got + kGuardBytes / 4, g.raw + kGuardBytes + g.bytes, kGuardBytes, cudaMemcpyDeviceToHost)))
+      return DMX_ERR_CUDA;
+    for (uint32_t w : got)
+      if (w != kGuardWord) return DMX_ERR_GUARD;
+  }
+  return DMX_OK;
+}
+
+int dmx_selftest_wait(dmx_handle* h, uint32_t polls, int* timed_out, double* waited_ms, void* cuda_stream) {
+  if (!live(h)) return DMX_ERR_HANDLE;
+  if (!timed_out || !waited_ms || polls < 1 || polls > (1u << 24)) return DMX_ERR_ARG;
+  if (const int rc = dmxh::check_current_device(h->device); rc != DMX_OK) return rc;
+  unsigned long long* d_out = nullptr;
+  if (!cuda_ok(cudaMalloc((void**)&d_out, 4 * sizeof(unsigned long long)))) return DMX_ERR_NOMEM;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  unsigned long long out[4] = {0, 0, 0, 0};
+  dmx::wait_selftest_kernel<<<1, 32, 0, stream>>>(h->flags + 1, polls, d_out);
+  const bool ok = cuda_ok(cudaGetLastError()) &&
+                  cuda_ok(cudaMemcpyAsync(out, d_out, sizeof(out), cudaMemcpyDeviceToHost, stream)) &&
+                  cuda_ok(cudaStreamSynchronize(stream));
+  cudaFree(d_out);
+  if (!ok) return DMX_ERR_CUDA;
+  *timed_out = (int)out[0];
+  *waited_ms = (double)out[2] * 1e-6;
+  return DMX_OK;
 }
 
 int dmx_destroy(dmx_handle* h) {
   if (!h) return DMX_OK;
-  if (h->magic != kMagic) return DMX_ERR_HANDLE;
+  if (!dmxh::live_remove(h, dmxh::kStepHandle)) return DMX_ERR_HANDLE;
   free_handle(h);
   return DMX_OK;
 }
@@ -684,6 +810,7 @@ const char* dmx_strerror(int code) {
     case DMX_ERR_CUDA: return "a CUDA runtime call failed";
     case DMX_ERR_HANDLE: return "invalid or destroyed handle";
     case DMX_ERR_LIMIT: return "problem exceeds the fixed scratch of dmx_step_static (too many segments)";
+    case DMX_ERR_GUARD: return "a guard word beside the handle's scratch was overwritten";
     default: return "unknown dmx error code";
   }
 }

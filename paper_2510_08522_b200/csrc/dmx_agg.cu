@@ -10,9 +10,9 @@
 #include <cuda_runtime.h>
 #include <new>
 
-namespace {
+#include "dmx_host.h"
 
-constexpr uint64_t kAggMagic = 0x444d585f41474752ull;  // "DMX_AGGR"
+namespace {
 
 __global__ void agg_push_kernel(const float* __restrict__ x, double* __restrict__ mean, double* __restrict__ m2,
                                 unsigned* __restrict__ flags_or, float* __restrict__ out, int len, int n, int k, int emit) {
@@ -46,7 +46,6 @@ __global__ void agg_push_kernel(const float* __restrict__ x, double* __restrict_
 }  // namespace
 
 struct dmx_agg {
-  uint64_t magic = kAggMagic;
   int len = 0, k = 0, n = 0;       // n: pushes into the current window so far
   double* mean = nullptr;
   double* m2 = nullptr;
@@ -59,32 +58,33 @@ int dmx_agg_create(int state_len, int k, dmx_agg** out) {
   if (!out) return DMX_ERR_ARG;
   *out = nullptr;
   if (state_len <= DMX_ST_FLAGS || k < 1) return DMX_ERR_ARG;
-  dmx_agg* a = new (std::nothrow) dmx_agg;
+  dmxh::alloc_begin();
+  dmx_agg* a = dmxh::alloc_host_ok() ? new (std::nothrow) dmx_agg : nullptr;
   if (!a) return DMX_ERR_NOMEM;
   a->len = state_len; a->k = k;
-  bool ok = cudaMalloc((void**)&a->mean, sizeof(double) * state_len) == cudaSuccess &&
-            cudaMalloc((void**)&a->m2, sizeof(double) * state_len) == cudaSuccess &&
-            cudaMalloc((void**)&a->flags_or, sizeof(unsigned)) == cudaSuccess;
+  const bool ok = dmxh::dev_alloc((void**)&a->mean, sizeof(double) * state_len) &&
+                  dmxh::dev_alloc((void**)&a->m2, sizeof(double) * state_len) &&
+                  dmxh::dev_alloc((void**)&a->flags_or, sizeof(unsigned));
   if (!ok) {
-    (void)cudaGetLastError();
     cudaFree(a->mean); cudaFree(a->m2); cudaFree(a->flags_or);
     (void)cudaGetLastError();
     delete a;
     return DMX_ERR_NOMEM;
   }
+  dmxh::live_add(a, dmxh::kAggHandle);
   *out = a;
   return DMX_OK;
 }
 
 int dmx_agg_push(dmx_agg* a, const float* out_state, float* window_out, int* emitted, void* cuda_stream) {
-  if (!a || a->magic != kAggMagic) return DMX_ERR_HANDLE;
+  if (!dmxh::live_has(a, dmxh::kAggHandle)) return DMX_ERR_HANDLE;
   if (!out_state || !window_out) return DMX_ERR_ARG;
   const int n = a->n + 1;
   const int emit = n == a->k ? 1 : 0;
   const int threads = 128, blocks = (a->len + threads - 1) / threads;
   agg_push_kernel<<<blocks, threads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(out_state, a->mean, a->m2, a->flags_or,
                                                                                 window_out, a->len, n, a->k, emit);
-  if (cudaGetLastError() != cudaSuccess) return DMX_ERR_CUDA;
+  if (!dmxh::cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
   a->n = emit ? 0 : n;
   if (emitted) *emitted = emit;
   return DMX_OK;
@@ -92,10 +92,9 @@ int dmx_agg_push(dmx_agg* a, const float* out_state, float* window_out, int* emi
 
 int dmx_agg_destroy(dmx_agg* a) {
   if (!a) return DMX_OK;
-  if (a->magic != kAggMagic) return DMX_ERR_HANDLE;
+  if (!dmxh::live_remove(a, dmxh::kAggHandle)) return DMX_ERR_HANDLE;
   cudaFree(a->mean); cudaFree(a->m2); cudaFree(a->flags_or);
   (void)cudaGetLastError();
-  a->magic = 0;
   delete a;
   return DMX_OK;
 }

@@ -75,6 +75,19 @@ __global__ void fill_kernel(void* __restrict__ dst, const float* __restrict__ ba
   }
 }
 
+// Number of SMs of the current device (asked once per device).
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 1;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
 int launch(void* dst, const float* base, float mean, float scale, int64_t n, int bf16,
            uint32_t seed, uint32_t tag, uint32_t c2, uint32_t c3, int accumulate, void* stream) {
   if (!dst || n < 1) return -1;
@@ -82,7 +95,8 @@ int launch(void* dst, const float* base, float mean, float scale, int64_t n, int
   if (!bf16 && (reinterpret_cast<uintptr_t>(dst) & 15)) return -4;
   const int threads = 256;
   int64_t blocks = ((n + 3) / 4 + threads - 1) / threads;
-  if (blocks > 148 * 64) blocks = 148 * 64;
+  const int64_t cap = (int64_t)sm_count() * 64;
+  if (blocks > cap) blocks = cap;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (bf16) fill_kernel<true><<<(unsigned)blocks, threads, 0, st>>>(dst, base, mean, scale, n, seed, tag, c2, c3, accumulate);
   else fill_kernel<false><<<(unsigned)blocks, threads, 0, st>>>(dst, base, mean, scale, n, seed, tag, c2, c3, accumulate);
@@ -115,7 +129,8 @@ __global__ void __launch_bounds__(256) read_probe_kernel(const __grid_constant__
 extern "C" {
 
 // Reads `bytes` bytes (a multiple of 16) of each of nsrc DEVICE buffers (16-byte aligned) once;
-// sink: DEVICE, at least 148 * 8 words, receives checksums. Returns 0 or a negative code.
+// sink: DEVICE, at least dmxgen_probe_sink_words() words (8 per SM of the current device), receives
+// checksums. Returns 0 or a negative code.
 int dmxgen_read_probe(const void* const* src, int nsrc, int64_t bytes, uint32_t* sink, void* stream) {
   if (!src || nsrc < 1 || nsrc > 64 || bytes < 16 || (bytes & 15) || !sink) return -1;
   ProbeArgs A;
@@ -124,9 +139,11 @@ int dmxgen_read_probe(const void* const* src, int nsrc, int64_t bytes, uint32_t*
     A.src[k] = static_cast<const uint4*>(src[k]);
   }
   A.nsrc = nsrc; A.n16 = bytes / 16; A.sink = sink;
-  read_probe_kernel<<<148 * 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(A);
+  read_probe_kernel<<<sm_count() * 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(A);
   return cudaGetLastError() == cudaSuccess ? 0 : -6;
 }
+
+int dmxgen_probe_sink_words(void) { return sm_count() * 8; }
 
 // dst[j] = mean + std * z_j                                  (fp32, DEVICE, 16-byte aligned)
 int dmxgen_normal_fill(float* dst, int64_t n, uint32_t seed, uint32_t tag, uint32_t c2, uint32_t c3,

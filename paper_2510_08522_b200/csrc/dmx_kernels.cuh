@@ -48,6 +48,24 @@ constexpr int kMaxK = 64;
 constexpr int kSegBuf = 32;                 // segment partials a CTA buffers in shared memory between drains
 constexpr int kTileBoundaryBit = 1 << 30;   // flag in the per-tile segment table
 
+// Error word of a handle: bit 0 = a bounded wait ran out, bit 1 = an index was out of range.
+constexpr unsigned kErrWait = 1u, kErrBounds = 2u;
+
+// Checked build (-DDMX_DEBUG): every index into the tables and the scratch is tested against its
+// range; a violation sets kErrBounds in the handle's error word (reported as DMX_FLAG_BOUNDS in
+// the state vector) and the access is skipped. Nothing traps. In the normal build the test
+// folds to `true`.
+#ifdef DMX_DEBUG
+__device__ __forceinline__ bool in_range(unsigned* err, long long i, long long n) {
+  if (i >= 0 && i < n) return true;
+  atomicOr(err, kErrBounds);
+  return false;
+}
+#define DMX_IN_RANGE(err, i, n) (::dmx::in_range((err), (long long)(i), (long long)(n)))
+#else
+#define DMX_IN_RANGE(err, i, n) (true)
+#endif
+
 // Arguments of one step; passed by value as a __grid_constant__ kernel parameter, so a step
 // needs no host-to-device copy. Worker arrays are in processing order (pivot first).
 struct StepArgs {
@@ -73,10 +91,13 @@ struct StepArgs {
   const int32_t* chunk_tile0;  // nchunks: first tile of the chunk
   const int32_t* chunk_ntiles; // nchunks: tiles in the chunk
   const int32_t* chunk_stride; // nchunks: tiles between the starts of the chunk's successive groups
-  const int32_t* chunk_slot0;  // nchunks: first (V,N) slot of the chunk
+  const int32_t* chunk_slot0;  // nchunks: index of the chunk's first (V,N) entry in slot_dest
+  const int32_t* slot_dest;    // nslots: where entry e of the step goes in `slots` (entries in the order the chunks emit them)
   float* rows;                 // (K+4) x nchunks, one column after the other: q_k..., c, pp, and (Adam) su, su2
-  float2* slots;               // nslots: (V partial, N partial), in the order the chunk emits them
-  unsigned* err;               // set non-zero when a bounded wait gives up
+  float2* slots;               // nslots: (V partial, N partial), grouped by segment, each group in entry order
+  unsigned* err;               // bit 0: a bounded wait gave up; bit 1 (checked build): an index was out of range
+  int ntiles, nslots;          // table sizes (range checks of the checked build)
+  int fold;                    // 1: the last CTA to finish runs the second level itself (one launch per step)
 };
 
 struct FinalArgs {
@@ -88,9 +109,10 @@ struct FinalArgs {
   double B;
   const float* rows;
   const float2* slots;
-  const int32_t* seg_slots;    // slot indices grouped by segment (each group in slot order)
-  const int32_t* unit_lo;      // nunits: a unit is a run seg_slots[unit_lo .. unit_hi) of one segment,
+  const int32_t* seg_ptr;      // S+1: the partials of segment s are slots[seg_ptr[s] .. seg_ptr[s+1])
+  const int32_t* unit_lo;      // nunits: a unit is a run slots[unit_lo .. unit_hi) of one segment,
   const int32_t* unit_hi;      //         at most kFinalPart slots long
+  int nslots;
   const int32_t* seg_unit_ptr; // S+1: units of segment s are [seg_unit_ptr[s], seg_unit_ptr[s+1])
   double2* segpart;            // nunits: (V, N) of each unit
   double* colsum;              // K+4
@@ -138,6 +160,15 @@ __device__ __forceinline__ u64 mul2(u64 a, u64 b) {
 __device__ __forceinline__ int tile_of(const StepArgs& A, int t0, int stride, int i) {
   const int g = i / A.tile_group;
   return t0 + g * stride + (i - g * A.tile_group);
+}
+
+// Processing order of a chunk's tiles: position i -> index of the tile within the chunk. A chunk
+// that ends with the ragged last tile of the problem takes that tile first: it is read with plain
+// loads (several dependent round trips to memory), and taken first that latency overlaps with
+// the bulk copies of the chunk's other tiles instead of following them. The host enumerates a
+// chunk's segment entries in the same order.
+__host__ __device__ __forceinline__ int chunk_order(int i, int nt, bool ragged_last) {
+  return ragged_last ? (i == 0 ? nt - 1 : i - 1) : i;
 }
 
 __device__ __forceinline__ float sqrt_approx(float x) { float r; asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
@@ -259,21 +290,25 @@ struct SegState {
 
 // Sum the buffered segment partials over the warps (fixed order) into their slots.
 template <int KT, int NW>
-__device__ __forceinline__ void seg_write(RedArea<KT, NW>* R, const SegState& st, float2* chunk_slots) {
+__device__ __forceinline__ void seg_write(RedArea<KT, NW>* R, const SegState& st, const StepArgs& A, int slot0) {
   for (int e = threadIdx.x; e < st.nbuf; e += NW * 32) {
     float v = 0.f, n = 0.f;
 #pragma unroll
     for (int w = 0; w < NW; ++w) { const float2 t = R->seg[st.par][e][w]; v += t.x; n += t.y; }
-    chunk_slots[st.nent - st.nbuf + e] = make_float2(v, n);
+    const int entry = slot0 + st.nent - st.nbuf + e;
+    if (DMX_IN_RANGE(A.err, entry, A.nslots)) {
+      const int dest = A.slot_dest[entry];
+      if (DMX_IN_RANGE(A.err, dest, A.nslots)) A.slots[dest] = make_float2(v, n);
+    }
   }
 }
 
 // The buffer is full in the middle of a chunk (more than kSegBuf segment boundaries in it):
 // empty it between two barriers.
 template <int KT, int NW, class SY>
-__device__ __forceinline__ void seg_drain(RedArea<KT, NW>* R, SegState& st, float2* chunk_slots, SY& sy) {
+__device__ __forceinline__ void seg_drain(RedArea<KT, NW>* R, SegState& st, const StepArgs& A, int slot0, SY& sy) {
   sy.sync();
-  seg_write<KT, NW>(R, st, chunk_slots);
+  seg_write<KT, NW>(R, st, A, slot0);
   sy.sync();
   st.nbuf = 0;
 }
@@ -281,13 +316,13 @@ __device__ __forceinline__ void seg_drain(RedArea<KT, NW>* R, SegState& st, floa
 // Close the running (vs, ns) as the next entry of the chunk: a warp reduction and one
 // shared-memory store per warp; no block barrier unless the shared buffer is full.
 template <int KT, int VEC, int NW, class SY>
-__device__ __forceinline__ void seg_entry(Acc<KT, VEC>& a, RedArea<KT, NW>* R, SegState& st, float2* chunk_slots,
+__device__ __forceinline__ void seg_entry(Acc<KT, VEC>& a, RedArea<KT, NW>* R, SegState& st, const StepArgs& A, int slot0,
                                           SY& sy, int wid, int lane) {
   const float v = warp_sum(a.vs), n = warp_sum(a.ns);
   if (lane == 0) R->seg[st.par][st.nbuf][wid] = make_float2(v, n);
   a.vs = 0.f; a.ns = 0.f;
   ++st.nbuf; ++st.nent;
-  if (st.nbuf == kSegBuf) seg_drain<KT, NW>(R, st, chunk_slots, sy);
+  if (st.nbuf == kSegBuf) seg_drain<KT, NW>(R, st, A, slot0, sy);
 }
 
 // Attribute the tile's per-element (d, g^2) to segments. `tseg` is the tile's table entry.
@@ -296,10 +331,10 @@ template <int KT, int VEC, int NW, class SY>
 __device__ __forceinline__ void segment_accumulate(Acc<KT, VEC>& a, const StepArgs& A, const float* dv,
                                                    const float* nv, int64_t jt, int64_t tile_begin,
                                                    int64_t tile_end, int tseg, RedArea<KT, NW>* R, SegState& st,
-                                                   float2* chunk_slots, SY& sy, int wid, int lane) {
+                                                   int slot0, SY& sy, int wid, int lane) {
   const int s0 = tseg & (kTileBoundaryBit - 1);
   if (s0 != st.cur) {
-    if (st.cur >= 0) seg_entry<KT, VEC, NW>(a, R, st, chunk_slots, sy, wid, lane);
+    if (st.cur >= 0) seg_entry<KT, VEC, NW>(a, R, st, A, slot0, sy, wid, lane);
     st.cur = s0;
   }
   if (!(tseg & kTileBoundaryBit)) {
@@ -315,7 +350,7 @@ __device__ __forceinline__ void segment_accumulate(Acc<KT, VEC>& a, const StepAr
       const int64_t j = jt + e;
       if (j >= lo && j < next_bound) { a.vs += dv[e]; a.ns += nv[e]; }
     }
-    seg_entry<KT, VEC, NW>(a, R, st, chunk_slots, sy, wid, lane);
+    seg_entry<KT, VEC, NW>(a, R, st, A, slot0, sy, wid, lane);
     lo = next_bound;
     ++st.cur;
     next_bound = A.seg_off[st.cur + 1];
@@ -330,8 +365,8 @@ __device__ __forceinline__ void segment_accumulate(Acc<KT, VEC>& a, const StepAr
 // the chunk's scratch row.
 template <int KT, int VEC, int NW, bool ADAM, class SY>
 __device__ __forceinline__ void flush_chunk(Acc<KT, VEC>& a, const StepArgs& A, RedArea<KT, NW>* R, SegState& st,
-                                            int chunk, float2* chunk_slots, SY& sy, int wid, int lane) {
-  if (st.cur >= 0) seg_entry<KT, VEC, NW>(a, R, st, chunk_slots, sy, wid, lane);
+                                            int chunk, int slot0, SY& sy, int wid, int lane) {
+  if (st.cur >= 0) seg_entry<KT, VEC, NW>(a, R, st, A, slot0, sy, wid, lane);
   constexpr int NV = KT + 2 + (ADAM ? 2 : 0);
   float v[NV];
 #pragma unroll
@@ -343,14 +378,16 @@ __device__ __forceinline__ void flush_chunk(Acc<KT, VEC>& a, const StepArgs& A, 
     for (int i = 0; i < NV; ++i) R->rows[st.par][wid][i] = v[i];
   }
   sy.sync();                                       // the chunk's only barrier: every warp's partials are in place
-  seg_write<KT, NW>(R, st, chunk_slots);
+  seg_write<KT, NW>(R, st, A, slot0);
   const int t = wid * 32 + lane;
   if (t < NV) {
     float s = 0.f;
 #pragma unroll
     for (int w = 0; w < NW; ++w) s += R->rows[st.par][w][t];
-    if (t < KT) { if (t < A.K) A.rows[(int64_t)t * A.nchunks + chunk] = s; }
-    else A.rows[(int64_t)(A.K + t - KT) * A.nchunks + chunk] = s;
+    if (DMX_IN_RANGE(A.err, chunk, A.nchunks)) {
+      if (t < KT) { if (t < A.K) A.rows[(int64_t)t * A.nchunks + chunk] = s; }
+      else A.rows[(int64_t)(A.K + t - KT) * A.nchunks + chunk] = s;
+    }
   }
   st.par ^= 1;                                     // the next chunk fills the other copy
   a.reset_chunk();
@@ -509,7 +546,7 @@ __device__ __noinline__ void ragged_tile(Acc<KT, Elem<BF16>::VEC>& a, const Step
 
 template <int KT, bool BF16, int NW, int U, bool ADAM>
 __global__ void __launch_bounds__(NW * 32)
-direct_kernel(const __grid_constant__ StepArgs A) {
+direct_kernel(const __grid_constant__ StepArgs A, const __grid_constant__ FinalArgs) {
   constexpr int VEC = Elem<BF16>::VEC;
   constexpr int T = NW * 32 * VEC;
   __shared__ RedArea<KT, NW> R;
@@ -521,10 +558,12 @@ direct_kernel(const __grid_constant__ StepArgs A) {
   // chunks are dealt statically here: chunk c belongs to CTA c mod grid
   for (int c = blockIdx.x; c < A.nchunks; c += gridDim.x) {
     const int t0 = A.chunk_tile0[c], nt = A.chunk_ntiles[c], cstride = A.chunk_stride[c];
-    float2* chunk_slots = A.slots + A.chunk_slot0[c];
+    const int slot0 = A.chunk_slot0[c];
+    const bool rl = A.P % T != 0 && tile_of(A, t0, cstride, nt - 1) == A.ntiles - 1;
     st.begin_chunk();
     for (int i = 0; i < nt; ++i) {
-      const int t = tile_of(A, t0, cstride, i);
+      const int t = tile_of(A, t0, cstride, chunk_order(i, nt, rl));
+      if (!DMX_IN_RANGE(A.err, t, A.ntiles)) continue;
       const int tseg = A.tile_seg[t];
       const int64_t tile_begin = (int64_t)t * T;
       const int64_t jt = tile_begin + (int64_t)threadIdx.x * VEC;
@@ -536,9 +575,9 @@ direct_kernel(const __grid_constant__ StepArgs A) {
         tile_end = A.P;
         direct_tile<KT, BF16, true, U, ADAM>(a, A, jt, dv, nv);
       }
-      segment_accumulate<KT, VEC, NW>(a, A, dv, nv, jt, tile_begin, tile_end, tseg, &R, st, chunk_slots, sy, wid, lane);
+      segment_accumulate<KT, VEC, NW>(a, A, dv, nv, jt, tile_begin, tile_end, tseg, &R, st, slot0, sy, wid, lane);
     }
-    flush_chunk<KT, VEC, NW, ADAM>(a, A, &R, st, c, chunk_slots, sy, wid, lane);
+    flush_chunk<KT, VEC, NW, ADAM>(a, A, &R, st, c, slot0, sy, wid, lane);
   }
 }
 
@@ -556,7 +595,7 @@ constexpr int kFinalWarps = 8;
 // The scalar part of the state vector from the step's reduced sums (the definitions of the state
 // layout): D = sum_s Vraw_s, A = sum_s N_s, Qw = sum_k b_k q_k, c = <g,a>, pp = |a|^2.
 __device__ __forceinline__ void emit_header(float* out, int K, double B, double D, double A, double Qw, double c, double pp,
-                                            bool nonfinite_q, bool internal, int adam, double su, double su2, double P) {
+                                            bool nonfinite_q, unsigned errbits, int adam, double su, double su2, double P) {
   int flags = 0;
   double trS = 0.0;
   if (K >= 2) trS = D / (double)(K - 1); else flags |= 8;
@@ -568,7 +607,8 @@ __device__ __forceinline__ void emit_header(float* out, int K, double B, double 
   const double sig2 = A > 0.0 ? trS / (B * A) : 0.0;
   const double sig = sqrt(sig2 > 0.0 ? sig2 : 0.0);
   if (nonfinite_q || !isfinite((float)A) || !isfinite((float)pp)) flags |= 1;
-  if (internal) flags |= 16;
+  if (errbits & kErrWait) flags |= 16;
+  if (errbits & kErrBounds) flags |= 32;
   out[0] = (float)B; out[1] = (float)A; out[2] = (float)trS; out[3] = (float)G2; out[4] = (float)gns;
   out[5] = (float)cosv; out[6] = (float)c; out[7] = (float)pp; out[8] = (float)sig2; out[9] = (float)sig;
   out[10] = (float)(Qw / B); out[11] = (float)flags;
@@ -621,17 +661,17 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
   } else {
     const int u = ((int)blockIdx.x - ncol) * kFinalWarps + wid;
     if (u < F.nunits) {
-      const int lo = F.unit_lo[u], hi = F.unit_hi[u];
+      int lo = F.unit_lo[u], hi = F.unit_hi[u];
+      if (!DMX_IN_RANGE(F.err, lo, F.nslots + 1) || !DMX_IN_RANGE(F.err, hi, F.nslots + 1)) hi = lo = 0;
       double v = 0.0, n = 0.0, v1 = 0.0, n1 = 0.0, v2 = 0.0, n2 = 0.0, v3 = 0.0, n3 = 0.0;
       int i = lo + lane;
-      for (; i + 96 < hi; i += 128) {          // four gathers in flight per lane; fixed summation order
-        const int i0 = F.seg_slots[i], i1 = F.seg_slots[i + 32], i2 = F.seg_slots[i + 64], i3 = F.seg_slots[i + 96];
-        const float2 t0 = F.slots[i0], t1 = F.slots[i1], t2 = F.slots[i2], t3 = F.slots[i3];
+      for (; i + 96 < hi; i += 128) {          // four loads in flight per lane; fixed summation order
+        const float2 t0 = F.slots[i], t1 = F.slots[i + 32], t2 = F.slots[i + 64], t3 = F.slots[i + 96];
         v += (double)t0.x; n += (double)t0.y; v1 += (double)t1.x; n1 += (double)t1.y;
         v2 += (double)t2.x; n2 += (double)t2.y; v3 += (double)t3.x; n3 += (double)t3.y;
       }
       for (; i < hi; i += 32) {
-        const float2 t = F.slots[F.seg_slots[i]];
+        const float2 t = F.slots[i];
         v += (double)t.x; n += (double)t.y;
       }
       v = warp_sum_d((v + v1) + (v2 + v3)); n = warp_sum_d((n + n1) + (n2 + n3));
@@ -668,9 +708,10 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
     if (threadIdx.x == 0) {
       pt[K] = cs[K]; pt[K + 1] = cs[K + 1];
       pt[K + 2] = F.adam ? cs[K + 2] : 0.0; pt[K + 3] = F.adam ? cs[K + 3] : 0.0;
-      const bool internal = *reinterpret_cast<volatile unsigned*>(F.err) != 0u;
-      pt[K + 4 + 2 * S] = internal ? 1.0 : 0.0;
-      if (internal) *F.err = 0u;
+      const unsigned errbits = *reinterpret_cast<volatile unsigned*>(F.err);
+      // summed over the shards: waits that ran out count 1 each, range violations 65536 each
+      pt[K + 4 + 2 * S] = (double)(errbits & kErrWait) + 65536.0 * (double)((errbits & kErrBounds) != 0u);
+      if (errbits) *F.err = 0u;
       *F.next_chunk = 0u;
       *F.ticket = 0u;
     }
@@ -694,9 +735,9 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
     for (int w = 0; w < kFinalWarps; ++w) { D += s_red[0][w]; A += s_red[1][w]; }
     bool bad = false;
     for (int k = 0; k < K; ++k) { const double qk = cs[k]; Qw += F.b[k] * qk; bad = bad | !isfinite((float)qk); }
-    const bool internal = *reinterpret_cast<volatile unsigned*>(F.err) != 0u;
-    if (internal) *F.err = 0u;
-    emit_header(out, K, F.B, D, A, Qw, cs[K], cs[K + 1], bad, internal, F.adam, F.adam ? cs[K + 2] : 0.0,
+    const unsigned errbits = *reinterpret_cast<volatile unsigned*>(F.err);
+    if (errbits) *F.err = 0u;
+    emit_header(out, K, F.B, D, A, Qw, cs[K], cs[K + 1], bad, errbits, F.adam, F.adam ? cs[K + 2] : 0.0,
                 F.adam ? cs[K + 3] : 0.0, F.P);
     *F.next_chunk = 0u;                      // the fused pass has completed: ready for the next step (or a graph replay)
     *F.ticket = 0u;
@@ -726,7 +767,126 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) derive_kernel(const _
     for (int w = 0; w < kFinalWarps; ++w) { D += s_red[0][w]; A += s_red[1][w]; }
     bool bad = false;
     for (int k = 0; k < K; ++k) { const double qk = pt[k]; Qw += G.b[k] * qk; bad = bad | !isfinite((float)qk); }
-    emit_header(out, K, G.B, D, A, Qw, pt[K], pt[K + 1], bad, pt[K + 4 + 2 * S] != 0.0, G.adam, pt[K + 2], pt[K + 3], G.P);
+    // the error words of the shards were added up: any wait that ran out, any index out of range
+    const double ew = pt[K + 4 + 2 * S];
+    const unsigned errbits = (fmod(ew, 65536.0) != 0.0 ? kErrWait : 0u) | (ew >= 65536.0 ? kErrBounds : 0u);
+    emit_header(out, K, G.B, D, A, Qw, pt[K], pt[K + 1], bad, errbits, G.adam, pt[K + 2], pt[K + 3], G.P);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Second level inside the fused pass, for problems whose scratch is small (a few hundred
+// chunks): the CTAs count themselves off on the ticket when their last chunk's partials are
+// written and fenced, and the NW warps of the one that counts last do the whole second level
+// out of shared memory. One launch per step instead of two: on a 100 us step the separate
+// finalize kernel costs 8-10 us behind the fused pass (its blocks' start-up, three dependent
+// trips to memory, a second ticket), this costs about half of that. A ticket is a count, not a
+// wait: no CTA waits for another. The sums are taken in a fixed order that does not depend on
+// which CTA is last, so results stay bitwise reproducible.
+//
+// Limits (checked by the host when it chooses this form): the chunk rows (ncol x nchunks
+// floats), the slots and the segment pointers must fit the work area below.
+constexpr int kFoldMaxRowFloats = 24576;   // 96 KB
+constexpr int kFoldMaxSlots = 4096;        // 32 KB
+constexpr int kFoldMaxSegments = 512;
+constexpr int kFoldParts = 8;              // a column is summed in this many runs, then the runs in order
+constexpr size_t kFoldWorkBytes = (size_t)kFoldMaxRowFloats * 4 + (size_t)kFoldMaxSlots * 8 + (kFoldMaxSegments + 4) * 4 +
+                                  (size_t)(kMaxK + 4) * (kFoldParts + 1) * 8 + (size_t)kFoldMaxSegments * 16 + 64 * 8;
+
+__device__ __forceinline__ float ldcg_f(const float* p) { float v; asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p)); return v; }
+__device__ __forceinline__ float2 ldcg_f2(const float2* p) {
+  float2 v; asm volatile("ld.global.cg.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p)); return v;
+}
+
+template <int NW, class SY>
+__device__ __noinline__ void fold_finalize(const FinalArgs& F, unsigned char* work, SY& sy, int wid, int lane) {
+  constexpr int NT = NW * 32;
+  const int tid = wid * 32 + lane;
+  const int K = F.K, S = F.S, nch = F.nchunks;
+  const int ncol = K + 2 + 2 * F.adam;
+  float* s_rows = reinterpret_cast<float*>(work);                                   // ncol x nch
+  float2* s_slots = reinterpret_cast<float2*>(s_rows + kFoldMaxRowFloats);          // nslots
+  int* s_ptr = reinterpret_cast<int*>(s_slots + kFoldMaxSlots);                     // S+1
+  double* s_part = reinterpret_cast<double*>(s_ptr + kFoldMaxSegments + 4);         // ncol x kFoldParts
+  double* s_cs = s_part + (kMaxK + 4) * kFoldParts;                                 // ncol
+  double2* s_seg = reinterpret_cast<double2*>(s_cs + kMaxK + 4);                    // S
+  double* s_red = reinterpret_cast<double*>(s_seg + kFoldMaxSegments);              // 2 x 32
+  // everything the other CTAs wrote, in one sweep of independent loads (served by L2)
+  const int nrow = ncol * nch;
+  for (int i = tid; i < nrow; i += NT) s_rows[i] = ldcg_f(F.rows + i);
+  for (int i = tid; i < F.nslots; i += NT) s_slots[i] = ldcg_f2(F.slots + i);
+  for (int i = tid; i <= S; i += NT) s_ptr[i] = F.seg_ptr[i];
+  sy.sync();
+  // column sums: run r of column c covers chunks [r per, (r+1) per)
+  const int per = (nch + kFoldParts - 1) / kFoldParts;
+  for (int p = tid; p < ncol * kFoldParts; p += NT) {
+    const int c = p / kFoldParts, r = p - c * kFoldParts;
+    const int lo = r * per, hi = lo + per < nch ? lo + per : nch;
+    const float* col = s_rows + c * nch;
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+    int i = lo;
+    for (; i + 3 < hi; i += 4) { a0 += (double)col[i]; a1 += (double)col[i + 1]; a2 += (double)col[i + 2]; a3 += (double)col[i + 3]; }
+    for (; i < hi; ++i) a0 += (double)col[i];
+    s_part[p] = (a0 + a1) + (a2 + a3);
+  }
+  // segment sums: eight lanes per segment, a fixed stride and a fixed shuffle tree
+  constexpr int NG = NT / 8;
+  const int grp = tid >> 3, gl = tid & 7;
+  for (int s0 = 0; s0 < S; s0 += NG) {            // uniform trip count: the shuffles below need whole warps
+    const int sidx = s0 + grp;
+    double v = 0.0, n = 0.0;
+    if (sidx < S) {
+      int lo = s_ptr[sidx], hi = s_ptr[sidx + 1];
+      if (!DMX_IN_RANGE(F.err, lo, F.nslots + 1) || !DMX_IN_RANGE(F.err, hi, F.nslots + 1)) hi = lo = 0;
+      for (int i = lo + gl; i < hi; i += 8) { const float2 t = s_slots[i]; v += (double)t.x; n += (double)t.y; }
+    }
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) { v += __shfl_xor_sync(0xffffffffu, v, o); n += __shfl_xor_sync(0xffffffffu, n, o); }
+    if (sidx < S && gl == 0) s_seg[sidx] = make_double2(v, n);
+  }
+  sy.sync();
+  if (tid < ncol) {
+    double t = 0.0;
+#pragma unroll
+    for (int r = 0; r < kFoldParts; ++r) t += s_part[tid * kFoldParts + r];
+    s_cs[tid] = t;
+  }
+  if (wid == NW - 1) {                             // D and A: lanes stride through the segments, then the tree
+    double aV = 0.0, aN = 0.0;
+    for (int s = lane; s < S; s += 32) { aV += s_seg[s].x; aN += s_seg[s].y; }
+    aV = warp_sum_d(aV); aN = warp_sum_d(aN);
+    if (lane == 0) { s_red[0] = aV; s_red[1] = aN; }
+  }
+  sy.sync();
+  if (F.partials) {
+    double* pt = F.partials;
+    for (int s = tid; s < S; s += NT) { pt[K + 4 + s] = s_seg[s].x; pt[K + 4 + S + s] = s_seg[s].y; }
+    for (int k = tid; k < K; k += NT) pt[F.orig[k]] = s_cs[k];
+  } else {
+    float* out = F.out_state;
+    for (int s = tid; s < S; s += NT) {
+      out[16 + K + s] = K >= 2 ? (float)(s_seg[s].x / (double)(K - 1)) : 0.f;
+      out[16 + K + S + s] = (float)s_seg[s].y;
+    }
+    for (int k = tid; k < K; k += NT) out[16 + F.orig[k]] = (float)s_cs[k];
+  }
+  if (tid == 0) {
+    const unsigned errbits = *reinterpret_cast<volatile unsigned*>(F.err);
+    if (errbits) *F.err = 0u;
+    if (F.partials) {
+      double* pt = F.partials;
+      pt[K] = s_cs[K]; pt[K + 1] = s_cs[K + 1];
+      pt[K + 2] = F.adam ? s_cs[K + 2] : 0.0; pt[K + 3] = F.adam ? s_cs[K + 3] : 0.0;
+      pt[K + 4 + 2 * S] = (double)(errbits & kErrWait) + 65536.0 * (double)((errbits & kErrBounds) != 0u);
+    } else {
+      double Qw = 0.0;
+      bool bad = false;
+      for (int k = 0; k < K; ++k) { const double qk = s_cs[k]; Qw += F.b[k] * qk; bad = bad | !isfinite((float)qk); }
+      emit_header(F.out_state, K, F.B, s_red[0], s_red[1], Qw, s_cs[K], s_cs[K + 1], bad, errbits, F.adam,
+                  F.adam ? s_cs[K + 2] : 0.0, F.adam ? s_cs[K + 3] : 0.0, F.P);
+    }
+    *F.next_chunk = 0u;                      // ready for the next step (or a graph replay)
+    *F.ticket = 0u;
   }
 }
 
@@ -762,10 +922,11 @@ constexpr uint32_t kWaitLimit = 1u << 24;
 
 // Bounded wait. Returns false (at once) when the CTA has given up, and raises the give-up
 // flag itself when its own polling budget runs out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* give_up, unsigned* err) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* give_up, unsigned* err,
+                                          uint32_t limit = kWaitLimit) {
   if (mbar_try_wait(bar, parity)) return true;
   if (*give_up) return false;
-  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 1023u) == 1023u && *give_up) return false;
   }
@@ -827,15 +988,16 @@ struct PipeCfg {
   static constexpr int RED = (int)((sizeof(RedArea<KT, CW>) + 15) / 16 * 16);
   static constexpr int QN = 4;                       // chunk descriptors in flight from the producer to the consumers
   static constexpr int NBAR = 2 * NSTAGE + 2 * NSS + 2 * QN + 1;
-  static constexpr int TAIL = 16 + QN * 32;          // give-up word, chunk queue (8 ints per entry)
+  static constexpr int TAIL = 16 + QN * 32;          // give-up word, last-CTA word, chunk queue (8 ints per entry)
   static constexpr size_t SMEM = (size_t)RING + SRING + RED + NBAR * 8 + TAIL;
   static_assert(G >= 1 && G <= 32, "one producer lane per stream of a stage");
   static_assert(NSTAGE <= 32 && NSS <= 32, "stage masks are 32 bits wide");
   static_assert(SMEM <= 227 * 1024, "ring does not fit in shared memory");
+  static_assert((size_t)RING + SRING >= kFoldWorkBytes, "the folded second level works in the ring's memory");
 };
 
 template <class C>
-__global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_constant__ StepArgs A) {
+__global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_constant__ StepArgs A, const __grid_constant__ FinalArgs F) {
   constexpr int KT = C::KT, VEC = C::VEC, CW = C::CW, G = C::G, NSTAGE = C::NSTAGE, NSS = C::NSS, T = C::T, QN = C::QN;
   constexpr bool BF16 = C::BF16, ADAM = C::ADAM;
   extern __shared__ __align__(128) unsigned char smem[];
@@ -845,6 +1007,7 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
   const uint32_t bars = sring + C::SRING + C::RED;
   unsigned char* tail = smem + C::RING + C::SRING + C::RED + C::NBAR * 8;
   volatile uint32_t* give_up = reinterpret_cast<volatile uint32_t*>(tail);
+  volatile uint32_t* is_last = reinterpret_cast<volatile uint32_t*>(tail + 4);
   volatile int* queue = reinterpret_cast<volatile int*>(tail + 16);   // entry: chunk (-1: none left), first tile,
                                                                        // tiles, group stride, first slot
   // barriers, 8 bytes each: full_g[NSTAGE], empty_g[NSTAGE], full_s[NSS], empty_s[NSS],
@@ -852,12 +1015,15 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
   const uint32_t full_g = bars, empty_g = bars + 8 * NSTAGE, full_s = bars + 16 * NSTAGE, empty_s = full_s + 8 * NSS;
   const uint32_t full_q = empty_s + 8 * NSS, empty_q = full_q + 8 * QN, csync = empty_q + 8 * QN;
   const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < NSTAGE; ++i) { mbar_init(full_g + 8 * i, 1); mbar_init(empty_g + 8 * i, CW); }
-    for (int i = 0; i < NSS; ++i) { mbar_init(full_s + 8 * i, 1); mbar_init(empty_s + 8 * i, CW); }
-    for (int i = 0; i < QN; ++i) { mbar_init(full_q + 8 * i, 1); mbar_init(empty_q + 8 * i, CW); }
-    mbar_init(csync, CW);
-    *give_up = 0u;
+  // one thread per barrier (a single thread initialising all of them in turn costs the CTA half a
+  // microsecond before its first copy): "full" barriers take one arrival, the others one per consumer warp
+  static_assert(C::NBAR <= C::THREADS, "one thread per barrier");
+  if ((int)threadIdx.x < C::NBAR) {
+    const int i = threadIdx.x;
+    const bool full = i < NSTAGE || (i >= 2 * NSTAGE && i < 2 * NSTAGE + NSS) ||
+                      (i >= 2 * NSTAGE + 2 * NSS && i < 2 * NSTAGE + 2 * NSS + QN);
+    mbar_init(bars + 8 * i, full ? 1 : CW);
+    if (i == 0) { *give_up = 0u; *is_last = 0u; }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -890,7 +1056,7 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
     while (ok) {
       ok = __all_sync(0xffffffffu, mbar_wait(empty_q + 8 * qi, qphase ^ 1u, give_up, A.err));
       if (!ok) break;
-      unsigned drawn = 0u;
+      unsigned drawn = 0xffffffffu;                              // no draw made: nothing more for this CTA
       if (lane == 0) {
         volatile int* e = queue + 8 * qi;
         e[0] = cur; e[1] = c_t0; e[2] = c_nt; e[3] = c_stride; e[4] = c_slot0;
@@ -902,10 +1068,13 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
       const int t0 = __shfl_sync(0xffffffffu, c_t0, 0), nt = __shfl_sync(0xffffffffu, c_nt, 0);
       const int cstride = __shfl_sync(0xffffffffu, c_stride, 0);
       const int draw_at = nt > 3 ? nt - 3 : 0;
+      const bool rl = A.P % T != 0 && tile_of(A, t0, cstride, nt - 1) == A.ntiles - 1;
       for (int i = 0; i < nt && ok; ++i) {
         if (lane == 0 && i == draw_at) drawn = atomicAdd(A.next_chunk, 1u) + gridDim.x;
-        const int64_t tile_begin = (int64_t)tile_of(A, t0, cstride, i) * T;
-        if (tile_begin + T > A.P) break;  // the ragged last tile is read with plain loads
+        const int t = tile_of(A, t0, cstride, chunk_order(i, nt, rl));
+        if (!DMX_IN_RANGE(A.err, t, A.ntiles)) continue;
+        const int64_t tile_begin = (int64_t)t * T;
+        if (tile_begin + T > A.P) continue;  // the ragged last tile is read by the consumers with plain loads
         for (int k0 = 0; k0 < A.K; k0 += G) {
           ok = __all_sync(0xffffffffu, mbar_wait(empty_g + 8 * stage, phase ^ 1u, give_up, A.err));
           if (!ok) break;
@@ -973,10 +1142,11 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
     if (lane == 0) mbar_arrive(empty_q + 8 * qi);
     if (++qi == QN) { qi = 0; qphase ^= 1u; }
     if (c < 0) break;
-    float2* chunk_slots = A.slots + slot0;
+    const bool rl = A.P % T != 0 && tile_of(A, t0, cstride, nt - 1) == A.ntiles - 1;
     st.begin_chunk();
     for (int i = 0; i < nt; ++i) {
-      const int t = tile_of(A, t0, cstride, i);
+      const int t = tile_of(A, t0, cstride, chunk_order(i, nt, rl));
+      if (!DMX_IN_RANGE(A.err, t, A.ntiles)) continue;
       const int tseg = A.tile_seg[t];          // needed only at the end of the tile: latency hidden
       const int64_t tile_begin = (int64_t)t * T;
       const int64_t jt = tile_begin + (int64_t)tid * VEC;
@@ -1040,9 +1210,48 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
 #pragma unroll
         for (int e = 0; e < VEC; ++e) { dv[e] = dv2[e]; nv[e] = nv2[e]; }
       }
-      segment_accumulate<KT, VEC, CW>(a, A, dv, nv, jt, tile_begin, tile_end, tseg, R, st, chunk_slots, sy, wid, lane);
+      segment_accumulate<KT, VEC, CW>(a, A, dv, nv, jt, tile_begin, tile_end, tseg, R, st, slot0, sy, wid, lane);
     }
-    flush_chunk<KT, VEC, CW, ADAM>(a, A, R, st, c, chunk_slots, sy, wid, lane);
+    flush_chunk<KT, VEC, CW, ADAM>(a, A, R, st, c, slot0, sy, wid, lane);
+  }
+  if (A.fold) {
+    // this CTA's partial sums are written: make them visible, count the CTA off, and if it is the
+    // last one of the grid, do the second level here (the ring is idle: every copy has landed)
+    __threadfence();
+    sy.sync();
+    if (tid == 0) *is_last = atomicAdd(F.ticket, 1u) == gridDim.x - 1 ? 1u : 0u;
+    sy.sync();
+    if (*is_last) {
+      __threadfence();
+      fold_finalize<CW>(F, smem, sy, wid, lane);
+    }
+  }
+}
+
+// Self-test of the bounded wait: one warp waits, with a polling budget of `limit`, on an
+// mbarrier that nothing will ever complete (no copy is in flight, nobody else arrives), so the
+// wait must run out: it raises the give-up word and the handle's error word exactly as a wait
+// of the fused pass would. out[0] = 1 if the wait reported failure, out[1] = the give-up word,
+// out[2..3] = nanoseconds spent in the wait (%globaltimer).
+static __global__ void __launch_bounds__(32) wait_selftest_kernel(unsigned* err, uint32_t limit, unsigned long long* out) {
+  __shared__ __align__(8) unsigned long long bar_storage;
+  __shared__ uint32_t give_up_word;
+  const uint32_t bar = smem_u32(&bar_storage);
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    give_up_word = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  unsigned long long t0, t1;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+  const bool ok = mbar_wait(bar, 0u, &give_up_word, err, limit);
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
+  __syncwarp();
+  if (threadIdx.x == 0) {
+    out[0] = ok ? 0ull : 1ull;
+    out[1] = (unsigned long long)give_up_word;
+    out[2] = t1 - t0;
   }
 }
 

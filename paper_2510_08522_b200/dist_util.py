@@ -10,33 +10,45 @@ from __future__ import annotations
 import os
 
 _world = 1
+_group = False      # a process group exists: the collectives run (always so when the world has more than one rank)
 
 
-def init(world: int, backend: str = "nccl") -> None:
-    """Join the process group described by RANK / WORLD_SIZE / MASTER_ADDR / MASTER_PORT."""
-    global _world
+def init(world: int, backend: str = "nccl", group_of_one: bool = False) -> None:
+    """Join the process group described by RANK / WORLD_SIZE / MASTER_ADDR / MASTER_PORT.
+    A world of one needs no group and every collective below is then the identity; with
+    `group_of_one` a one-rank group is created all the same and the collectives run through the
+    backend (how the nccl branches are exercised where only one GPU is available)."""
+    global _world, _group
     _world = int(world)
-    if _world <= 1:
+    _group = _world > 1 or group_of_one
+    if not _group:
         return
     import torch.distributed as dist
     os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
     if not dist.is_initialized():
-        dist.init_process_group(backend=backend, rank=int(os.environ["RANK"]), world_size=_world)
+        dist.init_process_group(backend=backend, rank=int(os.environ.get("RANK", "0")), world_size=_world)
+
+
+def _host_staged():
+    """gloo moves host memory: device tensors go through a host copy (tests on CPU or with
+    several processes on one GPU); nccl takes device tensors as they are."""
+    import torch.distributed as dist
+    return dist.get_backend() != "nccl"
 
 
 def barrier() -> None:
-    if _world > 1:
+    if _group:
         import torch.distributed as dist
         dist.barrier()
 
 
 def max_over_ranks(x: float) -> float:
     """Max of a per-rank scalar (timings are reported as the slowest rank's)."""
-    if _world <= 1:
+    if not _group:
         return float(x)
     import torch
     import torch.distributed as dist
-    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    dev = "cpu" if _host_staged() else "cuda"
     t = torch.tensor([float(x)], dtype=torch.float64, device=dev)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
@@ -45,9 +57,14 @@ def max_over_ranks(x: float) -> float:
 def allreduce_sum(t):
     """Entry-wise sum over the ranks of a tensor (the shards' partial sums), in place; the
     tensor lives where the backend wants it (device memory for nccl, host memory for gloo)."""
-    if _world > 1:
+    if _group:
         import torch.distributed as dist
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        if _host_staged() and t.is_cuda:
+            h = t.cpu()
+            dist.all_reduce(h, op=dist.ReduceOp.SUM)
+            t.copy_(h)
+        else:
+            dist.all_reduce(t, op=dist.ReduceOp.SUM)
     return t
 
 
@@ -77,28 +94,29 @@ def exchange_gradient_ranges(local_grad, ranges, rank: int):
     n = hi - lo
     stride = (n + 7) // 8 * 8
     out = torch.zeros((world, max(stride, 8)), dtype=local_grad.dtype, device=local_grad.device)
-    if world == 1:
+    if not _group:
         out[0, :n] = local_grad[lo:hi]
         return out
-    if dist.get_backend() == "nccl":
+    if not _host_staged():
         send = [local_grad[a:b] for a, b in ranges]
         recv = [out[k, :n] for k in range(world)]
         dist.all_to_all(recv, send)
     else:
-        full = [torch.empty_like(local_grad) for _ in range(world)]
-        dist.all_gather(full, local_grad.contiguous())
+        mine = local_grad.contiguous().cpu()
+        full = [torch.empty_like(mine) for _ in range(world)]
+        dist.all_gather(full, mine)
         for k in range(world):
-            out[k, :n] = full[k][lo:hi]
+            out[k, :n] = full[k][lo:hi].to(out.device)
     return out
 
 
 def gather_batch_sizes(b_local: int):
     """Every worker's batch size, in rank order (host ints)."""
-    if _world <= 1:
+    if not _group:
         return [int(b_local)]
     import torch
     import torch.distributed as dist
-    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    dev = "cpu" if _host_staged() else "cuda"
     mine = torch.tensor([int(b_local)], dtype=torch.int64, device=dev)
     every = [torch.zeros_like(mine) for _ in range(_world)]
     dist.all_gather(every, mine)
@@ -111,16 +129,17 @@ def allgather_ranges(shard, ranges, out_full):
     import torch
     import torch.distributed as dist
     world = len(ranges)
-    if world == 1:
+    if not _group:
         out_full[ranges[0][0]:ranges[0][1]] = shard[:ranges[0][1] - ranges[0][0]]
         return out_full
     longest = max(b - a for a, b in ranges)
-    mine = torch.zeros(longest, dtype=shard.dtype, device=shard.device)
+    staged = _host_staged() and shard.is_cuda
+    mine = torch.zeros(longest, dtype=shard.dtype, device="cpu" if staged else shard.device)
     mine[:shard.numel()] = shard
     every = [torch.empty_like(mine) for _ in range(world)]
     dist.all_gather(every, mine)
     for (a, b), t in zip(ranges, every):
-        out_full[a:b] = t[:b - a]
+        out_full[a:b] = t[:b - a].to(out_full.device)
     return out_full
 
 
@@ -148,10 +167,11 @@ def job_throughput(units_per_rank: float, local_ms: float) -> float:
 
 
 def finish() -> None:
-    global _world
-    if _world > 1:
+    global _world, _group
+    if _group:
         import torch.distributed as dist
         if dist.is_initialized():
             dist.barrier()
             dist.destroy_process_group()
     _world = 1
+    _group = False

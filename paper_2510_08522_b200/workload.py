@@ -274,7 +274,8 @@ def gen_lib():
         L.dmxgen_normal_add.argtypes = [vp, i64, u32, u32, u32, u32, f32, vp]
         L.dmxgen_grad_fill.argtypes = [vp, i32, vp, i64, u32, u32, u32, u32, f32, vp]
         L.dmxgen_read_probe.argtypes = [vp, i32, i64, vp, vp]
-        for f in (L.dmxgen_normal_fill, L.dmxgen_normal_add, L.dmxgen_grad_fill, L.dmxgen_read_probe):
+        L.dmxgen_probe_sink_words.argtypes = []
+        for f in (L.dmxgen_normal_fill, L.dmxgen_normal_add, L.dmxgen_grad_fill, L.dmxgen_read_probe, L.dmxgen_probe_sink_words):
             f.restype = i32
         _gen = L
     return _gen
@@ -353,7 +354,8 @@ def read_probe_gbps(tensors, reps=5):
     n = len(tensors)
     nbytes = min(t.numel() * t.element_size() for t in tensors) // 16 * 16
     ptrs = (ctypes.c_void_p * n)(*[t.data_ptr() for t in tensors])
-    sink = torch.zeros(148 * 8, dtype=torch.int32, device=tensors[0].device)
+    with torch.cuda.device(tensors[0].device):
+        sink = torch.zeros(L.dmxgen_probe_sink_words(), dtype=torch.int32, device=tensors[0].device)
     stream = torch.cuda.current_stream(tensors[0].device).cuda_stream
     ts = []
     for i in range(reps + 1):

@@ -15,6 +15,6 @@ def pytest_sessionstart(session):
     # cross-compiles without a GPU); a failure here is reported by the tests that load them
     try:
         from paper_2510_08522_b200 import build
-        build.build()
+        build.build(checked=True)
     except Exception as e:  # noqa: BLE001
         sys.stderr.write("conftest: building the CUDA libraries failed: %r\n" % (e,))

@@ -29,8 +29,9 @@ def cond_vectors(grads_f32, b, params_in, momentum_in, lr, beta):
     return cg, cm, ct
 
 
-def cond_vectors_adam(grads_f32, b, params_in, m_in, v_in, lr, beta1, beta2, eps, t):
-    """Forward-error scales of g, m', v', theta' under the Adam update (float64 arrays)."""
+def cond_vectors_adam(grads_f32, b, params_in, m_in, v_in, lr, beta1, beta2, eps, t, with_update=False):
+    """Forward-error scales of g, m', v', theta' under the Adam update (float64 arrays). With
+    with_update also |u| and the scale cu of the update u = mhat/(sqrt(vhat)+eps) itself."""
     w = np.asarray(b, np.float64) / float(np.sum(b))
     cg = np.zeros(len(params_in), np.float64)
     g = np.zeros(len(params_in), np.float64)
@@ -48,6 +49,8 @@ def cond_vectors_adam(grads_f32, b, params_in, m_in, v_in, lr, beta1, beta2, eps
     u = m_new * c1 / np.maximum(den, 1e-300)
     cu = c1 * cm / np.maximum(den, 1e-300) + np.abs(u) * c2 * cv / np.maximum(2 * root * den, 1e-300)
     ct = np.abs(params_in.astype(np.float64)) + abs(float(np.float32(lr))) * (np.abs(u) + cu)
+    if with_update:
+        return cg, cm, cv, ct, np.abs(u), cu
     return cg, cm, cv, ct
 
 
@@ -138,7 +141,8 @@ def check_state(gpu, ref, K, S, seg, b, what="", tol=TOL_S, seg_scale=None, adam
         rel(9, "sigma_norm", t=2 * tol)
     # flags: must match unless the reference sits on a threshold
     fg, fr = int(gpu[11]), int(ref[11])
-    assert not fg & 16, "%s internal-error flag set" % what
+    assert not fg & 16, "%s internal-error flag set (a bounded wait ran out)" % what
+    assert not fg & 32, "%s range-check flag set (checked build: an index was out of range)" % what
     mask = 1 | 4 | 8
     if abs(G2) > tol * max(A, 1e-300):
         mask |= 2

@@ -20,12 +20,13 @@ def declared_functions():
 
 
 def test_library_is_built_and_exports_every_declared_symbol():
-    build.build()
-    lib = ctypes.CDLL(build.lib_path("libdmx.so"))
+    build.build(checked=True)
     names = declared_functions()
     assert set(B.EXPORTS) <= set(names)
-    for n in names:
-        assert hasattr(lib, n), n
+    for so in ("libdmx.so", "libdmx_checked.so"):       # the checked build has the same ABI
+        lib = ctypes.CDLL(build.lib_path(so))
+        for n in names:
+            assert hasattr(lib, n), (so, n)
     gen = ctypes.CDLL(build.lib_path("libdmx_gen.so"))
     for n in ("dmxgen_normal_fill", "dmxgen_normal_add", "dmxgen_grad_fill", "dmxgen_read_probe"):
         assert hasattr(gen, n)
@@ -51,9 +52,29 @@ def test_create_rejects_bad_arguments_without_a_gpu():
     assert B.dmx_state_len(None) == B.ERR_HANDLE
     assert B.dmx_destroy(None) == B.OK
     assert B.dmx_step(None, [16], [1], 16, 32, 0.1, 0.9, 48, 64) == B.ERR_HANDLE
-    for code in range(-7, 1):
+    for code in range(-9, 1):
         assert D.strerror(code) and "unknown" not in D.strerror(code)
     assert "unknown" in D.strerror(-99)
+
+
+def test_a_pointer_that_is_not_a_live_handle_is_refused_without_being_read():
+    # handles are looked up in the table of live handles; an arbitrary (unmapped) address must come
+    # back as DMX_ERR_HANDLE from every entry point that takes a handle, not as a crash
+    bogus = ctypes.c_void_p(0x10)
+    assert B.dmx_state_len(bogus) == B.ERR_HANDLE
+    assert B.dmx_partials_len(bogus) == B.ERR_HANDLE
+    assert B.dmx_launches_per_step(bogus) == B.ERR_HANDLE
+    assert B.dmx_set_profiling(bogus, 1) == B.ERR_HANDLE
+    assert B.dmx_get_profile(bogus)[0] == B.ERR_HANDLE
+    assert B.dmx_check_guards(bogus) == B.ERR_HANDLE
+    assert B.dmx_selftest_wait(bogus, 16)[0] == B.ERR_HANDLE
+    assert B.dmx_step(bogus, [16], [1], 16, 32, 0.1, 0.9, 48, 64) == B.ERR_HANDLE
+    assert B.dmx_step_adam(bogus, [16], [1], 16, 32, 80, 0.1, 0.9, 0.99, 1e-8, 1, 48, 64) == B.ERR_HANDLE
+    assert B.dmx_step_partial(bogus, [16], [1], 16, 32, 0.1, 0.9, 48, 64) == B.ERR_HANDLE
+    assert B.dmx_step_host(bogus, [16], [16], [1], 16, 32, 0.1, 0.9, 48, 64, 80) == B.ERR_HANDLE
+    assert B.dmx_destroy(bogus) == B.ERR_HANDLE
+    assert B.dmx_agg_push(bogus, 16, 32)[0] == B.ERR_HANDLE
+    assert B.dmx_agg_destroy(bogus) == B.ERR_HANDLE
 
 
 def test_workload_tables():

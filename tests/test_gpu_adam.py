@@ -51,6 +51,62 @@ def lock_step_adam(wl, steps, v0=0.0):
     return worst
 
 
+ILL_CONDITIONED = 64.0     # an update whose forward-error scale exceeds this many units is sign-like
+
+
+def free_run_adam(wl, steps):
+    """Oracle and CUDA path each free-run the Adam step from the same initial state. g, m and v are
+    held to the per-step bounds (their recurrences contract). theta is a running sum of updates
+    u = mhat/(sqrt(vhat)+eps) computed with an approximate square root and reciprocal, so its bound
+    is the running sum of the per-step scales lr (|u| + cu); and where an aggregate cancels to
+    nearly zero while v is still small, u is sign-like (cu >> |u|: a last-bit difference in g flips
+    a whole unit step): those elements, found from the ORACLE's own numbers, are left out of the
+    comparison of theta from then on, counted, and must stay a vanishing fraction."""
+    torch = _torch()
+    import paper_2510_08522_b200 as D
+    dp = W.DeviceProblem(wl)
+    second = torch.zeros(wl.P, dtype=torch.float32, device="cuda")
+    orc = Oracle(wl.K, wl.P, dp.seg, wl.dtype)
+    d = D.Dmx(wl.K, wl.P, dp.seg, wl.dtype)
+    hp, hm, hv, ha = (x.cpu().numpy().copy() for x in (dp.params, dp.momentum, second, dp.prev_agg))
+    theta0 = np.abs(hp.astype(np.float64))
+    run_scale = np.zeros(wl.P)
+    masked = np.zeros(wl.P, dtype=bool)
+    tol = PT.TOL_V[wl.dtype]
+    worst = {}
+    for t in range(1, steps + 1):
+        b = dp.fill()
+        raw, wide = PT.grads_to_host(torch, dp.grads, wl.dtype)
+        cg, cm, cv, ct, au, cu = PT.cond_vectors_adam(wide, b, hp, hm, hv, LR, B1, B2, EPS, t, with_update=True)
+        masked |= cu > ILL_CONDITIONED
+        run_scale += abs(float(np.float32(LR))) * (au + cu)
+        ref = orc.step_adam(raw, b, hp, hm, hv, LR, B1, B2, EPS, t, ha, nthreads=NTHREADS)
+        st = d.step_adam(dp.grads, b, dp.params, dp.momentum, second, LR, B1, B2, EPS, t, dp.prev_agg)
+        torch.cuda.synchronize()
+        what = "%s adam free run step %d" % (wl.name, t)
+        e = {"agg": PT.vec_err(dp.prev_agg.cpu().numpy(), ha, cg), "first_moment": PT.vec_err(dp.momentum.cpu().numpy(), hm, cm),
+             "second_moment": PT.vec_err(second.cpu().numpy(), hv, cv)}
+        keep = ~masked
+        e["params"] = PT.vec_err(dp.params.cpu().numpy()[keep], hp[keep], (theta0 + run_scale)[keep])
+        for k, v in e.items():
+            assert v <= tol, "%s %s: max scaled error %.3e > %.1e" % (what, k, v, tol)
+            worst[k] = max(worst.get(k, 0.0), v)
+        # the statistics see the state of this step only (no accumulation): the usual bounds
+        worst["state"] = max(worst.get("state", 0.0), PT.check_state(st.cpu().numpy(), ref, wl.K, wl.S, dp.seg, b, what,
+                                                                     seg_scale=PT.seg_scales(cg, dp.seg), adam=True))
+        dp.advance()
+    d.close()
+    frac = masked.mean()
+    assert frac <= 1e-3, "%s: %.2e of the parameters ill-conditioned" % (wl.name, frac)
+    worst["masked_fraction"] = float(frac)
+    return worst
+
+
+@pytest.mark.parametrize("idx,P,steps", [(0, 262_147, 6), (1, 333_337, 20), (2, 401_239, 20), (3, 290_011, 10), (4, 523_777, 10)])
+def test_adam_free_running(idx, P, steps):
+    print(free_run_adam(W.WORKLOADS[idx].scaled(P=P, steps=steps), steps))
+
+
 @pytest.mark.parametrize("idx,P,steps", [(0, 262_147, 3), (1, 333_337, 8), (2, 401_239, 8), (3, 290_011, 4), (4, 523_777, 4)])
 def test_adam_scaled_workloads_multi_step(idx, P, steps):
     print(lock_step_adam(W.WORKLOADS[idx].scaled(P=P, steps=steps), steps))

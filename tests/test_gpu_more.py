@@ -230,13 +230,13 @@ def test_profiling_hooks():
     from paper_2510_08522_b200 import binding as B
     c = Custom(rnd(3, 4, 50_000), [32, 64, 96, 128], [0, 50_000])
     d = D.Dmx(c.K, c.P, c.seg, 0)
-    assert d.launches_per_step == 2 and B.dmx_launches_per_step(None) == B.ERR_HANDLE
+    assert d.launches_per_step in (1, 2) and B.dmx_launches_per_step(None) == B.ERR_HANDLE
     assert B.dmx_get_profile(d._h)[0] == B.ERR_ARG            # profiling is off
     d.set_profiling(True)
     assert B.dmx_get_profile(d._h)[0] == B.ERR_ARG            # on, but no step recorded yet
     st_on = d.step(c.d_grads, c.b, c.d_params, c.d_momentum, 0.1, 0.9, c.d_prev).clone()
     fused_ms, fin_ms = d.profile()
-    assert 0.0 < fused_ms < 50.0 and 0.0 < fin_ms < 50.0
+    assert 0.0 < fused_ms < 50.0 and 0.0 <= fin_ms < 50.0      # a one-launch step has no second kernel to time
     d.set_profiling(False)
     assert B.dmx_get_profile(d._h)[0] == B.ERR_ARG
     # timing on or off does not change results: rerun the same step from the same state without it
@@ -279,11 +279,13 @@ def test_random_problems_match_the_oracle(seed):
             h2 = np.abs(0.01 * rng.standard_normal(P)).astype(np.float32)
             d2 = torch.from_numpy(h2.copy()).cuda()
             conds = PT.cond_vectors_adam(c.wide, c.b, c.params, c.momentum, h2, 1e-3, 0.9, 0.999, 1e-8, 3)
-            Oracle(K, P, c.seg, dtype).step_adam(c.raw, c.b, c.params, c.momentum, h2, 1e-3, 0.9, 0.999, 1e-8, 3, c.prev)
+            st_ref = Oracle(K, P, c.seg, dtype).step_adam(c.raw, c.b, c.params, c.momentum, h2, 1e-3, 0.9, 0.999, 1e-8, 3, c.prev)
             d = D.Dmx(K, P, c.seg, dtype)
             st = d.step_adam(c.d_grads, c.b, c.d_params, c.d_momentum, d2, 1e-3, 0.9, 0.999, 1e-8, 3, c.d_prev)
             torch.cuda.synchronize()
+            d.check_guards()
             d.close()
+            PT.check_state(st.cpu().numpy(), st_ref, K, S, c.seg, c.b, what, seg_scale=PT.seg_scales(conds[0], c.seg), adam=True)
             PT.check_vectors_adam(dtype, (c.d_prev.cpu().numpy(), c.d_momentum.cpu().numpy(), d2.cpu().numpy(), c.d_params.cpu().numpy()),
                                   (c.prev, c.momentum, h2, c.params), conds, what)
             assert int(st[11].item()) & 16 == 0, what

@@ -57,6 +57,7 @@ class Custom:
         st = d.step(self.d_grads, self.b, self.d_params, self.d_momentum, self.lr, self.beta, self.d_prev)
         _torch().cuda.synchronize()
         st_gpu = st.cpu().numpy()
+        d.check_guards()
         d.close()
         gpu = (self.d_prev.cpu().numpy(), self.d_momentum.cpu().numpy(), self.d_params.cpu().numpy())
         if check:
@@ -98,6 +99,7 @@ def free_run(wl, steps, every=1):
             for k, v in e.items():
                 worst[k] = max(worst.get(k, 0.0), v)
         dp.advance()
+    d.check_guards()
     d.close()
     return worst
 
@@ -117,54 +119,8 @@ def test_scaled_workloads_multi_step(idx, P, steps):
     print(idx, "worst errors", w)
 
 
-def test_cfg1_full_size_many_steps():
-    wl = W.WORKLOADS[1]
-    w = free_run(wl.scaled(P=wl.P, steps=20), 20, every=5)
-    print("cfg1 worst errors", w)
-
-
-def streamed_step(wl, nsteps=1, span=4 << 20):
-    """Full-size parity with the gradients streamed to the host in element ranges."""
-    torch, D = _torch(), _dmx()
-    dp = W.DeviceProblem(wl)
-    orc = Oracle(wl.K, wl.P, dp.seg, wl.dtype)
-    d = D.Dmx(wl.K, wl.P, dp.seg, wl.dtype)
-    worst = {}
-    for t in range(nsteps):
-        b = dp.fill()
-        in_params, in_mom, in_prev = dp.params.clone(), dp.momentum.clone(), dp.prev_agg.clone()
-        st = d.step(dp.grads, b, dp.params, dp.momentum, wl.lr, wl.beta, dp.prev_agg)
-        torch.cuda.synchronize()
-        orc.begin(b, wl.lr, wl.beta)
-        errs = {"agg": 0.0, "momentum": 0.0, "params": 0.0}
-        scale = np.zeros(wl.S)
-        for lo in range(0, wl.P, span):
-            hi = min(wl.P, lo + span)
-            raw, wide = PT.grads_to_host(torch, dp.grads, wl.dtype, lo, hi)
-            hp, hm, hv = (x[lo:hi].cpu().numpy() for x in (in_params, in_mom, in_prev))
-            conds = PT.cond_vectors(wide, b, hp, hm, wl.lr, wl.beta)
-            scale += PT.seg_scales(conds[0], dp.seg, lo)
-            orc.range(lo, raw, hp, hm, hv, nthreads=NTHREADS)
-            gpu = tuple(x[lo:hi].cpu().numpy() for x in (dp.prev_agg, dp.momentum, dp.params))
-            e = PT.check_vectors(wl.dtype, gpu, (hv, hm, hp), conds, "%s [%d,%d)" % (wl.name, lo, hi))
-            for k, v in e.items():
-                errs[k] = max(errs[k], v)
-        st_ref = orc.end()
-        errs["state"] = PT.check_state(st.cpu().numpy(), st_ref, wl.K, wl.S, dp.seg, b, wl.name, seg_scale=scale)
-        for k, v in errs.items():
-            worst[k] = max(worst.get(k, 0.0), v)
-        del in_params, in_mom, in_prev
-        dp.advance()
-    d.close()
-    return worst
-
-
-@pytest.mark.parametrize("idx,nsteps", [(2, 3), (3, 1), (4, 1)])
-def test_full_size_streamed(idx, nsteps):
-    # whole steps at the full size, in the launch configuration the benchmark times (the mid-sized
-    # workload for three steps, so that momentum and the previous aggregate are non-trivial too)
-    w = streamed_step(W.WORKLOADS[idx], nsteps)
-    print(idx, "worst errors", w)
+# The five workloads at their full sizes and full step counts, free-running, are in
+# tests/test_gpu_stated_steps.py.
 
 
 # ---- edge cases --------------------------------------------------------------------------------

@@ -66,6 +66,27 @@ def test_shares_shrink_towards_the_end_and_are_even(P, K, dtype, tile, ctas):
         assert share.max() <= 1.15 * share.mean() + 2 * R
 
 
+@pytest.mark.parametrize("group,chunk,min_kb", [(1, 4, 48), (2, 8, 0), (4, 64, 384), (8, 16, 0), (16, 128, 0), (3, 5, 1)])
+@pytest.mark.parametrize("P,K,dtype,tile,ctas", CASES[1:5] + CASES[7:12])
+def test_tuning_knobs_keep_the_list_valid(monkeypatch, group, chunk, min_kb, P, K, dtype, tile, ctas):
+    # what the kernel relies on, whatever the knobs: every chunk has at least one tile, every tile
+    # is in exactly one chunk, and a ragged last tile is the last tile of the first chunk
+    monkeypatch.setenv("DMX_TILE_GROUP", str(group))
+    monkeypatch.setenv("DMX_CHUNK_TILES", str(chunk))
+    if min_kb:
+        monkeypatch.setenv("DMX_MIN_CHUNK_KB", str(min_kb))
+    n, t0, nt, st, R, grid = D.dmx_plan_chunks(P, K, dtype, tile, ctas)
+    ntiles = -(-P // tile)
+    assert n > 0 and R == group and min(nt) >= 1
+    seen = np.zeros(ntiles, dtype=np.int32)
+    for c in range(n):
+        t = tiles_of(t0[c], nt[c], st[c], R)
+        np.add.at(seen, t, 1)
+        if P % tile and ntiles - 1 in t:
+            assert c == 0 and t[-1] == ntiles - 1
+    assert np.all(seen == 1)
+
+
 def test_plan_rejects_bad_arguments():
     assert D.dmx_plan_chunks(0, 4, B.F32, 896, 148)[0] == B.ERR_ARG
     assert D.dmx_plan_chunks(10, 0, B.F32, 896, 148)[0] == B.ERR_ARG
@@ -85,7 +106,7 @@ def test_random_problems_are_always_tiled_exactly():
         tile = 896 if dtype == B.F32 else 1792
         n, t0, nt, stv, R, grid = D.dmx_plan_chunks(P, K, dtype, tile, ctas)
         ntiles = -(-P // tile)
-        assert n > 0 and 1 <= grid <= ctas and sum(nt) == ntiles and max(nt) <= 32
+        assert n > 0 and 1 <= grid <= ctas and sum(nt) == ntiles and max(nt) <= 32 and min(nt) >= 1
         seen = np.zeros(ntiles, dtype=np.int32)
         for c in range(n):
             np.add.at(seen, tiles_of(t0[c], nt[c], stv[c], R), 1)

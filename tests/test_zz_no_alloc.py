@@ -3,13 +3,17 @@ framework allocator owns it all, or an allocation's device-wide synchronisation 
 affordable where the step runs). It must give the same step as dmx_step, to rounding: the two
 differ only in the order of their sums. Checked through the C ABI on two calls in a row (the
 second call finds the first call's leftovers in the shared scratch array), then on a problem of
-another shape, then at the size limit.
+another shape, then at the size limit; and against the CPU oracle itself on the shapes its
+kernel table and its segment search have to get right (one worker, more than 32 workers, empty
+segments, a boundary exactly on a tile edge, 512 segments on a full grid, and a 32-worker bf16
+problem of 32 Mi parameters, where every thread's partial sums run over its CTA's whole range).
 
 Collected last on purpose: a failure here leaves every other test already run.
 """
 import numpy as np
 import pytest
 
+from oracle.dmx_oracle import Oracle
 from paper_2510_08522_b200 import workload as W
 from tests import parity as PT
 
@@ -80,3 +84,66 @@ def test_static_rejects_what_does_not_fit():
     assert call([0, P], b=(1, 0)) == B.ERR_BATCH
     assert call([0, P]) == B.OK
     torch.cuda.synchronize()
+
+
+def static_against_oracle(K, P, seg, dtype, b, calls=2, seed=0, on_device=False):
+    """dmx_step_static and the oracle free-run from the same state over `calls` steps."""
+    torch, B = _setup()
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+    gdt = torch.float32 if dtype == 0 else torch.bfloat16
+    seg = np.asarray(seg, np.int64)
+    S = len(seg) - 1
+    mu = 0.1 * torch.randn(P, device="cuda", generator=gen)
+    st = [0.05 * torch.randn(P, device="cuda", generator=gen), torch.zeros(P, device="cuda"), torch.zeros(P, device="cuda")]
+    h = [t.cpu().numpy().copy() for t in st]
+    out = torch.full((16 + K + 2 * S,), 7.0, device="cuda")
+    orc = Oracle(K, P, seg, dtype)
+    for call in range(calls):
+        grads = [(mu + torch.randn(P, device="cuda", generator=gen) / float(np.sqrt(b[k]))).to(gdt) for k in range(K)]
+        raw, wide = PT.grads_to_host(torch, grads, dtype)
+        what = "static K=%d P=%d S=%d dtype=%d call %d" % (K, P, S, dtype, call)
+        if on_device:
+            cg, cm, ct = PT.cond_vectors_t(torch, grads, b, torch.from_numpy(h[0]).cuda(), torch.from_numpy(h[1]).cuda(), 0.1, 0.9)
+            scale = PT.seg_scales_t(torch, cg, seg)
+        else:
+            cg, cm, ct = PT.cond_vectors(wide, b, h[0], h[1], 0.1, 0.9)
+            scale = PT.seg_scales(cg, seg)
+        del wide
+        st_ref = orc.step(raw, b, h[0], h[1], 0.1, 0.9, h[2], nthreads=16)
+        assert B.dmx_step_static(K, P, seg, dtype, [g.data_ptr() for g in grads], b, st[0].data_ptr(), st[1].data_ptr(), 0.1, 0.9,
+                                 st[2].data_ptr(), out.data_ptr(), torch.cuda.current_stream().cuda_stream) == B.OK
+        torch.cuda.synchronize()
+        if on_device:
+            for name, gpu, ref, cond in (("agg", st[2], h[2], cg), ("momentum", st[1], h[1], cm), ("params", st[0], h[0], ct)):
+                e = PT.vec_err_t(torch, gpu, torch.from_numpy(ref).cuda(), cond)
+                assert e <= PT.TOL_V[dtype], "%s %s: max scaled error %.3e" % (what, name, e)
+        else:
+            PT.check_vectors(dtype, (st[2].cpu().numpy(), st[1].cpu().numpy(), st[0].cpu().numpy()), (h[2], h[1], h[0]), (cg, cm, ct), what)
+        PT.check_state(out.cpu().numpy(), st_ref, K, S, seg, b, what, seg_scale=scale)
+        del grads, raw
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_static_against_the_oracle_on_the_shapes_its_kernel_table_covers(dtype):
+    tile = 1024 if dtype == 0 else 2048          # elements per tile of the static path's kernel
+    static_against_oracle(1, 5 * tile + 3, [0, 7, 5 * tile + 3], dtype, [48], seed=1)                       # one worker: no spread
+    static_against_oracle(40, 3 * tile + 1, [0, tile, 3 * tile + 1], dtype, [16 * (1 + k % 5) for k in range(40)], seed=2)  # 64-slot kernel
+    P = 200 * tile + 5
+    seg = [0, 0, 3, 3, 3, tile, 2 * tile, 2 * tile, 7 * tile + 1, 150 * tile, 150 * tile, P, P]               # empty segments, boundaries on tile edges
+    static_against_oracle(5, P, seg, dtype, [32, 64, 96, 128, 160], seed=3)
+
+
+def test_static_at_the_limit_that_just_fits():
+    # 512 segments on a full grid: the per-CTA segment cells take 148 x 512 x 8 bytes of the 1 MiB array
+    torch, B = _setup()
+    P = 400 * 1024 + 77
+    rng = np.random.default_rng(5)
+    seg = np.concatenate([[0], np.sort(rng.integers(0, P + 1, B.STATIC_MAX_SEGMENTS - 1)), [P]])
+    static_against_oracle(6, P, seg, 0, [32, 64, 96, 128, 160, 192], seed=4)
+
+
+def test_static_k32_bf16_at_32_mi_parameters():
+    # the sizes the library is for: each thread's fp32 partials (q_k, c, pp, the segment sums) run over about nine
+    # thousand elements per worker here, and the 1e-4 bound on the scalars has to hold all the same
+    wl = W.WORKLOADS[4].scaled(P=(32 << 20) + 13)
+    static_against_oracle(wl.K, wl.P, wl.segment_table(), wl.dtype, [int(v) for v in wl.batch_sizes(0)], calls=2, seed=6, on_device=True)
