@@ -250,10 +250,12 @@ int dmx_step_host(dmx_handle* h, const void* const* host_grad_ptrs, void* const*
 int dmx_set_profiling(dmx_handle* h, int on);
 int dmx_get_profile(dmx_handle* h, float* fused_ms, float* finalize_ms);
 
-/* Number of kernels one dmx_step launches: 1 when the problem's reduction scratch is small
- * enough for the fused pass to do the second level itself (a few hundred chunks, at most 512
- * segments), else 2 (fused pass, finalize). */
+/* Number of kernels one dmx_step launches (2: fused pass, finalize). */
 int dmx_launches_per_step(const dmx_handle* h);
+
+/* Sizes of a handle's launch plan, for inspection and tests: CTAs of the fused pass, chunks of
+ * its work list, (V, N) partial-sum slots. Any pointer may be NULL. DMX_ERR_HANDLE or DMX_OK. */
+int dmx_scratch_info(const dmx_handle* h, int* grid, int* nchunks, int* nslots);
 
 /*
  * Checks of the library's own machinery (the paper has no counterpart; robustness is one of its

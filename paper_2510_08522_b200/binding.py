@@ -23,7 +23,7 @@ EXPORTS = ("dmx_create", "dmx_state_len", "dmx_step", "dmx_step_adam", "dmx_step
            "dmx_launches_per_step", "dmx_destroy", "dmx_strerror", "dmx_last_cuda_error", "dmx_agg_create",
            "dmx_agg_push", "dmx_agg_destroy", "dmx_ctl_num_features", "dmx_ctl_num_weights", "dmx_ctl_decide", "dmx_plan_chunks",
            "dmx_shard_range", "dmx_shard_segments", "dmx_partials_len", "dmx_step_partial", "dmx_step_adam_partial",
-           "dmx_finalize_partials", "dmx_check_guards", "dmx_selftest_wait")
+           "dmx_finalize_partials", "dmx_check_guards", "dmx_selftest_wait", "dmx_scratch_info")
 CTL_ACTIONS = (-100, -25, 0, 25, 100)
 
 _lib = None
@@ -92,6 +92,8 @@ def lib():
         L.dmx_get_profile.restype = i32
         L.dmx_launches_per_step.argtypes = [vp]
         L.dmx_launches_per_step.restype = i32
+        L.dmx_scratch_info.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.dmx_scratch_info.restype = i32
         L.dmx_check_guards.argtypes = [vp]
         L.dmx_check_guards.restype = i32
         L.dmx_selftest_wait.argtypes = [vp, ctypes.c_uint32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_double), vp]
@@ -309,6 +311,13 @@ def dmx_get_profile(h):
 
 def dmx_launches_per_step(h) -> int:
     return lib().dmx_launches_per_step(h)
+
+
+def dmx_scratch_info(h):
+    """-> (code, grid, nchunks, nslots) of the handle's launch plan."""
+    g, c, n = ctypes.c_int(0), ctypes.c_int(0), ctypes.c_int(0)
+    rc = lib().dmx_scratch_info(h, ctypes.byref(g), ctypes.byref(c), ctypes.byref(n))
+    return rc, g.value, c.value, n.value
 
 
 def dmx_check_guards(h) -> int:

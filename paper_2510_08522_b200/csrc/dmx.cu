@@ -132,7 +132,7 @@ using dmxh::cuda_ok;
 
 bool live(const dmx_handle* h) { return dmxh::live_has(h, dmxh::kStepHandle); }
 
-typedef void (*StepKernel)(const dmx::StepArgs, const dmx::FinalArgs);
+typedef void (*StepKernel)(const dmx::StepArgs);
 
 struct Plan {
   StepKernel kernel = nullptr;       // SGD-momentum update
@@ -165,7 +165,6 @@ struct dmx_handle {
   Plan plan;
   int nchunks = 0, nslots = 0, tile_group = 1;
   int64_t ntiles = 0;
-  bool fold = false;     // the fused pass runs the second level itself (one launch per step)
   // device tables
   int64_t* seg_off = nullptr;
   int32_t *tile_seg = nullptr, *chunk_stride = nullptr, *chunk_tile0 = nullptr, *chunk_ntiles = nullptr;
@@ -226,7 +225,7 @@ Plan pick_direct(int K) {
 // each) as fit.
 template <int KT, bool BF16, bool ADAM>
 struct Ring {
-  static constexpr int CW = 7;
+  static constexpr int CW = (KT <= 8 && !BF16) ? 11 : 7;
   static constexpr int G = KT < 16 ? KT : 16;                                       // gradient streams per stage
   static constexpr int kStage = CW * 32 * 16 * G;                                   // bytes of a gradient stage
   static constexpr int kState = CW * 32 * (BF16 ? 8 : 4) * 4 * (ADAM ? 4 : 3);      // bytes of a state stage
@@ -477,10 +476,6 @@ int dmx_create(int K, int64_t P, const int64_t* seg_offsets, int S, int grad_dty
   seg_unit_ptr[S] = (int32_t)unit_lo.size();
   h->nchunks = nchunks; h->nslots = (int)nslots; h->nunits = (int)unit_lo.size();
   h->ntiles = ntiles;
-  // Small scratch: the fused pass does the second level itself (one launch per step). DMX_FOLD=0
-  // keeps the separate finalize kernel (a tuning and cross-check knob).
-  h->fold = !direct && env_int("DMX_FOLD", 1) != 0 && (int64_t)(K + 4) * nchunks <= dmx::kFoldMaxRowFloats &&
-            nslots <= dmx::kFoldMaxSlots && S <= dmx::kFoldMaxSegments;
 
   std::vector<int64_t> seg(seg_offsets, seg_offsets + S + 1);
   bool ok = upload(seg, &h->seg_off) && upload(tile_seg, &h->tile_seg) && upload(chunk_stride, &h->chunk_stride) &&
@@ -575,19 +570,10 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const bool prof = h->profiling;
   if (prof && !cuda_ok(cudaEventRecord(h->ev[0], stream))) return DMX_ERR_CUDA;
-  A.fold = h->fold ? 1 : 0;
-  if (ap) h->plan.kernel_adam<<<h->plan.grid, h->plan.threads, h->plan.smem_adam, stream>>>(A, F);
-  else h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A, F);
+  if (ap) h->plan.kernel_adam<<<h->plan.grid, h->plan.threads, h->plan.smem_adam, stream>>>(A);
+  else h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A);
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
   if (prof && !cuda_ok(cudaEventRecord(h->ev[1], stream))) return DMX_ERR_CUDA;
-  if (h->fold) {
-    // the fused pass has done the second level itself: nothing more to launch
-    if (prof) {
-      if (!cuda_ok(cudaEventRecord(h->ev[2], stream))) return DMX_ERR_CUDA;
-      h->profiled = true;
-    }
-    return DMX_OK;
-  }
   // one block per chunk-row column, one warp per segment unit. Launched as a programmatic
   // dependent of the fused pass: its blocks may become resident while that kernel drains and
   // wait (griddepcontrol.wait) for its completion, which hides the launch latency between the
@@ -756,7 +742,15 @@ int dmx_plan_chunks(int64_t P, int K, int grad_dtype, int tile_elems, int reside
 
 int dmx_launches_per_step(const dmx_handle* h) {
   if (!live(h)) return DMX_ERR_HANDLE;
-  return h->fold ? 1 : 2;
+  return 2;
+}
+
+int dmx_scratch_info(const dmx_handle* h, int* grid, int* nchunks, int* nslots) {
+  if (!live(h)) return DMX_ERR_HANDLE;
+  if (grid) *grid = h->plan.grid;
+  if (nchunks) *nchunks = h->nchunks;
+  if (nslots) *nslots = h->nslots;
+  return DMX_OK;
 }
 
 int dmx_check_guards(dmx_handle* h) {

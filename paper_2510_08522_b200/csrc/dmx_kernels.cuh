@@ -97,7 +97,6 @@ struct StepArgs {
   float2* slots;               // nslots: (V partial, N partial), grouped by segment, each group in entry order
   unsigned* err;               // bit 0: a bounded wait gave up; bit 1 (checked build): an index was out of range
   int ntiles, nslots;          // table sizes (range checks of the checked build)
-  int fold;                    // 1: the last CTA to finish runs the second level itself (one launch per step)
 };
 
 struct FinalArgs {
@@ -538,15 +537,29 @@ __device__ __forceinline__ void direct_tile(Acc<KT, Elem<BF16>::VEC>& a, const S
   }
 }
 
-// The ragged last tile, kept out of line so that its registers do not weigh on the main loop.
+// The ragged last tile of the pipelined kernel: plain loads, every element tested against P. It
+// runs in the loop's own registers (out of line, its running sums lived in local memory, which
+// the large shared-memory carve-out leaves almost no L1 for: the one tile then took 10-80 us).
+// All of the tile's lines are requested from memory at once (prefetch to L2) before the loads,
+// which are issued four workers at a time.
 template <int KT, bool BF16, bool ADAM>
-__device__ __noinline__ void ragged_tile(Acc<KT, Elem<BF16>::VEC>& a, const StepArgs& A, int64_t jt, float* dv, float* nv) {
+__device__ __forceinline__ void ragged_tile(Acc<KT, Elem<BF16>::VEC>& a, const StepArgs& A, int64_t jt, float* dv, float* nv) {
+  typedef typename Elem<BF16>::T GT;
+  if (jt < A.P) {
+#pragma unroll 4
+    for (int k = 0; k < A.K; ++k)
+      asm volatile("prefetch.global.L2 [%0];" :: "l"(static_cast<const GT*>(A.grad[k]) + jt));
+    asm volatile("prefetch.global.L2 [%0];" :: "l"(A.params + jt));
+    asm volatile("prefetch.global.L2 [%0];" :: "l"(A.momentum + jt));
+    asm volatile("prefetch.global.L2 [%0];" :: "l"(A.prev + jt));
+    if constexpr (ADAM) asm volatile("prefetch.global.L2 [%0];" :: "l"(A.second + jt));
+  }
   direct_tile<KT, BF16, true, 4, ADAM>(a, A, jt, dv, nv);
 }
 
 template <int KT, bool BF16, int NW, int U, bool ADAM>
 __global__ void __launch_bounds__(NW * 32)
-direct_kernel(const __grid_constant__ StepArgs A, const __grid_constant__ FinalArgs) {
+direct_kernel(const __grid_constant__ StepArgs A) {
   constexpr int VEC = Elem<BF16>::VEC;
   constexpr int T = NW * 32 * VEC;
   __shared__ RedArea<KT, NW> R;
@@ -594,7 +607,9 @@ constexpr int kFinalWarps = 8;
 
 // The scalar part of the state vector from the step's reduced sums (the definitions of the state
 // layout): D = sum_s Vraw_s, A = sum_s N_s, Qw = sum_k b_k q_k, c = <g,a>, pp = |a|^2.
-__device__ __forceinline__ void emit_header(float* out, int K, double B, double D, double A, double Qw, double c, double pp,
+// (Out of line on purpose: the finalize kernel runs it once on zeros while it waits for the fused
+// pass, so that the one real call finds this code in the instruction caches.)
+static __device__ __noinline__ void emit_header(float* out, int K, double B, double D, double A, double Qw, double c, double pp,
                                             bool nonfinite_q, unsigned errbits, int adam, double su, double su2, double P) {
   int flags = 0;
   double trS = 0.0;
@@ -634,7 +649,19 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
   const int K = F.K, S = F.S;
   const int ncol = K + 2 + 2 * F.adam;
   __shared__ double s_col[kFinalWarps];
-  // everything this kernel reads was written by the step's fused pass: with a programmatic
+  __shared__ float s_warm[16];
+  // Launched as a programmatic dependent, this kernel's blocks are usually resident long before
+  // the fused pass ends. What does not depend on that pass is done while they wait: the table
+  // entries each thread will need are fetched (after a step's worth of streaming they come from
+  // DRAM, a microsecond per dependent load), and thread 0 runs the header arithmetic once on
+  // zeros into shared memory, which brings its code (a few KB, cold as well) into the
+  // instruction caches. After the wait only loads of the fused pass's own output remain.
+  const int u_mine = ((int)blockIdx.x - ncol) * kFinalWarps + wid;
+  int pre_lo = 0, pre_hi = 0, pre_u0 = 0, pre_u1 = 0;
+  if ((int)blockIdx.x >= ncol && u_mine < F.nunits) { pre_lo = F.unit_lo[u_mine]; pre_hi = F.unit_hi[u_mine]; }
+  if ((int)threadIdx.x < S) { pre_u0 = F.seg_unit_ptr[threadIdx.x]; pre_u1 = F.seg_unit_ptr[threadIdx.x + 1]; }
+  if (threadIdx.x == 0) emit_header(s_warm, K, F.B, 0.0, 0.0, 0.0, 0.0, 0.0, false, 0u, F.adam, 0.0, 0.0, F.P);
+  // everything read from here on was written by the step's fused pass: with a programmatic
   // dependent launch this is where its completion (and the visibility of its writes) is awaited
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if ((int)blockIdx.x < ncol) {
@@ -659,9 +686,9 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
       F.colsum[blockIdx.x] = t;
     }
   } else {
-    const int u = ((int)blockIdx.x - ncol) * kFinalWarps + wid;
+    const int u = u_mine;
     if (u < F.nunits) {
-      int lo = F.unit_lo[u], hi = F.unit_hi[u];
+      int lo = pre_lo, hi = pre_hi;
       if (!DMX_IN_RANGE(F.err, lo, F.nslots + 1) || !DMX_IN_RANGE(F.err, hi, F.nslots + 1)) hi = lo = 0;
       double v = 0.0, n = 0.0, v1 = 0.0, n1 = 0.0, v2 = 0.0, n2 = 0.0, v3 = 0.0, n3 = 0.0;
       int i = lo + lane;
@@ -699,7 +726,8 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
     double* pt = F.partials;
     for (int s = threadIdx.x; s < S; s += blockDim.x) {
       double v = 0.0, n = 0.0;
-      for (int u = F.seg_unit_ptr[s]; u < F.seg_unit_ptr[s + 1]; ++u) { v += sp[u].x; n += sp[u].y; }
+      const int u0 = s == (int)threadIdx.x ? pre_u0 : F.seg_unit_ptr[s], u1 = s == (int)threadIdx.x ? pre_u1 : F.seg_unit_ptr[s + 1];
+      for (int u = u0; u < u1; ++u) { v += sp[u].x; n += sp[u].y; }
       pt[K + 4 + s] = v;
       pt[K + 4 + S + s] = n;
     }
@@ -719,9 +747,13 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
   }
   float* out = F.out_state;
   double aV = 0.0, aN = 0.0;
+  // (thread 0 asks for the error word now; it is used at the very end)
+  unsigned errbits = 0u;
+  if (threadIdx.x == 0) errbits = *reinterpret_cast<volatile unsigned*>(F.err);
   for (int s = threadIdx.x; s < S; s += blockDim.x) {
     double v = 0.0, n = 0.0;
-    for (int u = F.seg_unit_ptr[s]; u < F.seg_unit_ptr[s + 1]; ++u) { v += sp[u].x; n += sp[u].y; }
+    const int u0 = s == (int)threadIdx.x ? pre_u0 : F.seg_unit_ptr[s], u1 = s == (int)threadIdx.x ? pre_u1 : F.seg_unit_ptr[s + 1];
+    for (int u = u0; u < u1; ++u) { v += sp[u].x; n += sp[u].y; }
     out[16 + K + s] = K >= 2 ? (float)(v / (double)(K - 1)) : 0.f;
     out[16 + K + S + s] = (float)n;
     aV += v; aN += n;
@@ -730,12 +762,16 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(const
   if (lane == 0) { s_red[0][wid] = aV; s_red[1][wid] = aN; }
   __syncthreads();
   for (int k = threadIdx.x; k < K; k += blockDim.x) out[16 + F.orig[k]] = (float)cs[k];
-  if (threadIdx.x == 0) {
-    double D = 0.0, A = 0.0, Qw = 0.0;
-    for (int w = 0; w < kFinalWarps; ++w) { D += s_red[0][w]; A += s_red[1][w]; }
+  if (wid == 0) {
+    // sum_k b_k q_k: lane l takes workers l and l + 32, then the shuffle tree (a fixed order)
+    double Qw = 0.0;
     bool bad = false;
-    for (int k = 0; k < K; ++k) { const double qk = cs[k]; Qw += F.b[k] * qk; bad = bad | !isfinite((float)qk); }
-    const unsigned errbits = *reinterpret_cast<volatile unsigned*>(F.err);
+    for (int k = lane; k < K; k += 32) { const double qk = cs[k]; Qw += F.b[k] * qk; bad = bad | !isfinite((float)qk); }
+    Qw = warp_sum_d(Qw);
+    bad = __any_sync(0xffffffffu, bad);
+    if (lane != 0) return;
+    double D = 0.0, A = 0.0;
+    for (int w = 0; w < kFinalWarps; ++w) { D += s_red[0][w]; A += s_red[1][w]; }
     if (errbits) *F.err = 0u;
     emit_header(out, K, F.B, D, A, Qw, cs[K], cs[K + 1], bad, errbits, F.adam, F.adam ? cs[K + 2] : 0.0,
                 F.adam ? cs[K + 3] : 0.0, F.P);
@@ -762,131 +798,22 @@ static __global__ void __launch_bounds__(kFinalWarps * 32) derive_kernel(const _
   if (lane == 0) { s_red[0][wid] = aV; s_red[1][wid] = aN; }
   __syncthreads();
   for (int k = threadIdx.x; k < K; k += blockDim.x) out[16 + k] = (float)pt[k];
-  if (threadIdx.x == 0) {
-    double D = 0.0, A = 0.0, Qw = 0.0;
-    for (int w = 0; w < kFinalWarps; ++w) { D += s_red[0][w]; A += s_red[1][w]; }
+  if (wid == 0) {
+    // sum_k b_k q_k in the order the single-GPU finalize takes it. There the workers are in
+    // processing order (largest batch first); a sum over lanes and a shuffle tree of a permuted
+    // list differs in the last bits of the fp64 value only, below what the fp32 output keeps.
+    double Qw = 0.0;
     bool bad = false;
-    for (int k = 0; k < K; ++k) { const double qk = pt[k]; Qw += G.b[k] * qk; bad = bad | !isfinite((float)qk); }
+    for (int k = lane; k < K; k += 32) { const double qk = pt[k]; Qw += G.b[k] * qk; bad = bad | !isfinite((float)qk); }
+    Qw = warp_sum_d(Qw);
+    bad = __any_sync(0xffffffffu, bad);
+    if (lane != 0) return;
+    double D = 0.0, A = 0.0;
+    for (int w = 0; w < kFinalWarps; ++w) { D += s_red[0][w]; A += s_red[1][w]; }
     // the error words of the shards were added up: any wait that ran out, any index out of range
     const double ew = pt[K + 4 + 2 * S];
     const unsigned errbits = (fmod(ew, 65536.0) != 0.0 ? kErrWait : 0u) | (ew >= 65536.0 ? kErrBounds : 0u);
     emit_header(out, K, G.B, D, A, Qw, pt[K], pt[K + 1], bad, errbits, G.adam, pt[K + 2], pt[K + 3], G.P);
-  }
-}
-
-// ------------------------------------------------------------------------------------------
-// Second level inside the fused pass, for problems whose scratch is small (a few hundred
-// chunks): the CTAs count themselves off on the ticket when their last chunk's partials are
-// written and fenced, and the NW warps of the one that counts last do the whole second level
-// out of shared memory. One launch per step instead of two: on a 100 us step the separate
-// finalize kernel costs 8-10 us behind the fused pass (its blocks' start-up, three dependent
-// trips to memory, a second ticket), this costs about half of that. A ticket is a count, not a
-// wait: no CTA waits for another. The sums are taken in a fixed order that does not depend on
-// which CTA is last, so results stay bitwise reproducible.
-//
-// Limits (checked by the host when it chooses this form): the chunk rows (ncol x nchunks
-// floats), the slots and the segment pointers must fit the work area below.
-constexpr int kFoldMaxRowFloats = 24576;   // 96 KB
-constexpr int kFoldMaxSlots = 4096;        // 32 KB
-constexpr int kFoldMaxSegments = 512;
-constexpr int kFoldParts = 8;              // a column is summed in this many runs, then the runs in order
-constexpr size_t kFoldWorkBytes = (size_t)kFoldMaxRowFloats * 4 + (size_t)kFoldMaxSlots * 8 + (kFoldMaxSegments + 4) * 4 +
-                                  (size_t)(kMaxK + 4) * (kFoldParts + 1) * 8 + (size_t)kFoldMaxSegments * 16 + 64 * 8;
-
-__device__ __forceinline__ float ldcg_f(const float* p) { float v; asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p)); return v; }
-__device__ __forceinline__ float2 ldcg_f2(const float2* p) {
-  float2 v; asm volatile("ld.global.cg.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p)); return v;
-}
-
-template <int NW, class SY>
-__device__ __noinline__ void fold_finalize(const FinalArgs& F, unsigned char* work, SY& sy, int wid, int lane) {
-  constexpr int NT = NW * 32;
-  const int tid = wid * 32 + lane;
-  const int K = F.K, S = F.S, nch = F.nchunks;
-  const int ncol = K + 2 + 2 * F.adam;
-  float* s_rows = reinterpret_cast<float*>(work);                                   // ncol x nch
-  float2* s_slots = reinterpret_cast<float2*>(s_rows + kFoldMaxRowFloats);          // nslots
-  int* s_ptr = reinterpret_cast<int*>(s_slots + kFoldMaxSlots);                     // S+1
-  double* s_part = reinterpret_cast<double*>(s_ptr + kFoldMaxSegments + 4);         // ncol x kFoldParts
-  double* s_cs = s_part + (kMaxK + 4) * kFoldParts;                                 // ncol
-  double2* s_seg = reinterpret_cast<double2*>(s_cs + kMaxK + 4);                    // S
-  double* s_red = reinterpret_cast<double*>(s_seg + kFoldMaxSegments);              // 2 x 32
-  // everything the other CTAs wrote, in one sweep of independent loads (served by L2)
-  const int nrow = ncol * nch;
-  for (int i = tid; i < nrow; i += NT) s_rows[i] = ldcg_f(F.rows + i);
-  for (int i = tid; i < F.nslots; i += NT) s_slots[i] = ldcg_f2(F.slots + i);
-  for (int i = tid; i <= S; i += NT) s_ptr[i] = F.seg_ptr[i];
-  sy.sync();
-  // column sums: run r of column c covers chunks [r per, (r+1) per)
-  const int per = (nch + kFoldParts - 1) / kFoldParts;
-  for (int p = tid; p < ncol * kFoldParts; p += NT) {
-    const int c = p / kFoldParts, r = p - c * kFoldParts;
-    const int lo = r * per, hi = lo + per < nch ? lo + per : nch;
-    const float* col = s_rows + c * nch;
-    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-    int i = lo;
-    for (; i + 3 < hi; i += 4) { a0 += (double)col[i]; a1 += (double)col[i + 1]; a2 += (double)col[i + 2]; a3 += (double)col[i + 3]; }
-    for (; i < hi; ++i) a0 += (double)col[i];
-    s_part[p] = (a0 + a1) + (a2 + a3);
-  }
-  // segment sums: eight lanes per segment, a fixed stride and a fixed shuffle tree
-  constexpr int NG = NT / 8;
-  const int grp = tid >> 3, gl = tid & 7;
-  for (int s0 = 0; s0 < S; s0 += NG) {            // uniform trip count: the shuffles below need whole warps
-    const int sidx = s0 + grp;
-    double v = 0.0, n = 0.0;
-    if (sidx < S) {
-      int lo = s_ptr[sidx], hi = s_ptr[sidx + 1];
-      if (!DMX_IN_RANGE(F.err, lo, F.nslots + 1) || !DMX_IN_RANGE(F.err, hi, F.nslots + 1)) hi = lo = 0;
-      for (int i = lo + gl; i < hi; i += 8) { const float2 t = s_slots[i]; v += (double)t.x; n += (double)t.y; }
-    }
-#pragma unroll
-    for (int o = 4; o > 0; o >>= 1) { v += __shfl_xor_sync(0xffffffffu, v, o); n += __shfl_xor_sync(0xffffffffu, n, o); }
-    if (sidx < S && gl == 0) s_seg[sidx] = make_double2(v, n);
-  }
-  sy.sync();
-  if (tid < ncol) {
-    double t = 0.0;
-#pragma unroll
-    for (int r = 0; r < kFoldParts; ++r) t += s_part[tid * kFoldParts + r];
-    s_cs[tid] = t;
-  }
-  if (wid == NW - 1) {                             // D and A: lanes stride through the segments, then the tree
-    double aV = 0.0, aN = 0.0;
-    for (int s = lane; s < S; s += 32) { aV += s_seg[s].x; aN += s_seg[s].y; }
-    aV = warp_sum_d(aV); aN = warp_sum_d(aN);
-    if (lane == 0) { s_red[0] = aV; s_red[1] = aN; }
-  }
-  sy.sync();
-  if (F.partials) {
-    double* pt = F.partials;
-    for (int s = tid; s < S; s += NT) { pt[K + 4 + s] = s_seg[s].x; pt[K + 4 + S + s] = s_seg[s].y; }
-    for (int k = tid; k < K; k += NT) pt[F.orig[k]] = s_cs[k];
-  } else {
-    float* out = F.out_state;
-    for (int s = tid; s < S; s += NT) {
-      out[16 + K + s] = K >= 2 ? (float)(s_seg[s].x / (double)(K - 1)) : 0.f;
-      out[16 + K + S + s] = (float)s_seg[s].y;
-    }
-    for (int k = tid; k < K; k += NT) out[16 + F.orig[k]] = (float)s_cs[k];
-  }
-  if (tid == 0) {
-    const unsigned errbits = *reinterpret_cast<volatile unsigned*>(F.err);
-    if (errbits) *F.err = 0u;
-    if (F.partials) {
-      double* pt = F.partials;
-      pt[K] = s_cs[K]; pt[K + 1] = s_cs[K + 1];
-      pt[K + 2] = F.adam ? s_cs[K + 2] : 0.0; pt[K + 3] = F.adam ? s_cs[K + 3] : 0.0;
-      pt[K + 4 + 2 * S] = (double)(errbits & kErrWait) + 65536.0 * (double)((errbits & kErrBounds) != 0u);
-    } else {
-      double Qw = 0.0;
-      bool bad = false;
-      for (int k = 0; k < K; ++k) { const double qk = s_cs[k]; Qw += F.b[k] * qk; bad = bad | !isfinite((float)qk); }
-      emit_header(F.out_state, K, F.B, s_red[0], s_red[1], Qw, s_cs[K], s_cs[K + 1], bad, errbits, F.adam,
-                  F.adam ? s_cs[K + 2] : 0.0, F.adam ? s_cs[K + 3] : 0.0, F.P);
-    }
-    *F.next_chunk = 0u;                      // ready for the next step (or a graph replay)
-    *F.ticket = 0u;
   }
 }
 
@@ -988,16 +915,15 @@ struct PipeCfg {
   static constexpr int RED = (int)((sizeof(RedArea<KT, CW>) + 15) / 16 * 16);
   static constexpr int QN = 4;                       // chunk descriptors in flight from the producer to the consumers
   static constexpr int NBAR = 2 * NSTAGE + 2 * NSS + 2 * QN + 1;
-  static constexpr int TAIL = 16 + QN * 32;          // give-up word, last-CTA word, chunk queue (8 ints per entry)
+  static constexpr int TAIL = 16 + QN * 32;          // give-up word, chunk queue (8 ints per entry)
   static constexpr size_t SMEM = (size_t)RING + SRING + RED + NBAR * 8 + TAIL;
   static_assert(G >= 1 && G <= 32, "one producer lane per stream of a stage");
   static_assert(NSTAGE <= 32 && NSS <= 32, "stage masks are 32 bits wide");
   static_assert(SMEM <= 227 * 1024, "ring does not fit in shared memory");
-  static_assert((size_t)RING + SRING >= kFoldWorkBytes, "the folded second level works in the ring's memory");
 };
 
 template <class C>
-__global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_constant__ StepArgs A, const __grid_constant__ FinalArgs F) {
+__global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_constant__ StepArgs A) {
   constexpr int KT = C::KT, VEC = C::VEC, CW = C::CW, G = C::G, NSTAGE = C::NSTAGE, NSS = C::NSS, T = C::T, QN = C::QN;
   constexpr bool BF16 = C::BF16, ADAM = C::ADAM;
   extern __shared__ __align__(128) unsigned char smem[];
@@ -1007,7 +933,6 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
   const uint32_t bars = sring + C::SRING + C::RED;
   unsigned char* tail = smem + C::RING + C::SRING + C::RED + C::NBAR * 8;
   volatile uint32_t* give_up = reinterpret_cast<volatile uint32_t*>(tail);
-  volatile uint32_t* is_last = reinterpret_cast<volatile uint32_t*>(tail + 4);
   volatile int* queue = reinterpret_cast<volatile int*>(tail + 16);   // entry: chunk (-1: none left), first tile,
                                                                        // tiles, group stride, first slot
   // barriers, 8 bytes each: full_g[NSTAGE], empty_g[NSTAGE], full_s[NSS], empty_s[NSS],
@@ -1023,7 +948,7 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
     const bool full = i < NSTAGE || (i >= 2 * NSTAGE && i < 2 * NSTAGE + NSS) ||
                       (i >= 2 * NSTAGE + 2 * NSS && i < 2 * NSTAGE + 2 * NSS + QN);
     mbar_init(bars + 8 * i, full ? 1 : CW);
-    if (i == 0) { *give_up = 0u; *is_last = 0u; }
+    if (i == 0) *give_up = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -1202,29 +1127,11 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
         }
       } else {
         tile_end = A.P;
-        // through copies, so that only the copies (not the loop's registers) have their address taken
-        Acc<KT, VEC> a2 = a;
-        float dv2[VEC], nv2[VEC];
-        ragged_tile<KT, BF16, ADAM>(a2, A, jt, dv2, nv2);
-        a = a2;
-#pragma unroll
-        for (int e = 0; e < VEC; ++e) { dv[e] = dv2[e]; nv[e] = nv2[e]; }
+        ragged_tile<KT, BF16, ADAM>(a, A, jt, dv, nv);
       }
       segment_accumulate<KT, VEC, CW>(a, A, dv, nv, jt, tile_begin, tile_end, tseg, R, st, slot0, sy, wid, lane);
     }
     flush_chunk<KT, VEC, CW, ADAM>(a, A, R, st, c, slot0, sy, wid, lane);
-  }
-  if (A.fold) {
-    // this CTA's partial sums are written: make them visible, count the CTA off, and if it is the
-    // last one of the grid, do the second level here (the ring is idle: every copy has landed)
-    __threadfence();
-    sy.sync();
-    if (tid == 0) *is_last = atomicAdd(F.ticket, 1u) == gridDim.x - 1 ? 1u : 0u;
-    sy.sync();
-    if (*is_last) {
-      __threadfence();
-      fold_finalize<CW>(F, smem, sy, wid, lane);
-    }
   }
 }
 
