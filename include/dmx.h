@@ -269,7 +269,8 @@ int dmx_scratch_info(const dmx_handle* h, int* grid, int* nchunks, int* nslots);
  * dmx_selftest_wait — every wait inside the fused pass is bounded: after a fixed number of polls
  *   it gives up, raises the handle's error word and the CTA drains; the step's state vector then
  *   carries DMX_FLAG_INTERNAL and the word is cleared for the next step. This launches one warp
- *   that waits, with a budget of `polls` (1..2^24) polls, on a barrier that nothing will ever
+ *   that waits, with a budget of `polls` (1..2^24; the fused pass itself uses 2^18, about one
+ *   second on B200 at 4 us per unsuccessful poll) polls, on a barrier that nothing will ever
  *   complete (no copy in flight, nobody to arrive): the wait must run out. *timed_out (HOST)
  *   receives 1 if it did; *waited_ms (HOST) the time the warp spent waiting, by the GPU's timer.
  *   The handle's error word is raised exactly as by a failed wait in a step: the next step of the
