@@ -537,13 +537,18 @@ __device__ __forceinline__ void direct_tile(Acc<KT, Elem<BF16>::VEC>& a, const S
   }
 }
 
-// The ragged last tile of the pipelined kernel: plain loads, every element tested against P. It
-// runs in the loop's own registers (out of line, its running sums lived in local memory, which
-// the large shared-memory carve-out leaves almost no L1 for: the one tile then took 10-80 us).
+// The ragged last tile of the pipelined kernel: plain loads, every element tested against P.
 // All of the tile's lines are requested from memory at once (prefetch to L2) before the loads,
-// which are issued four workers at a time.
+// which are issued four workers at a time. Two forms, chosen by the kernel's worker capacity:
+//  - in the loop's own registers (few workers). Out of line, the running sums live in local
+//    memory, which the large shared-memory carve-out leaves almost no L1 for: the one tile then
+//    took 10-80 us, a large part of a step of a few million parameters.
+//  - out of line, on copies (many workers). Inlined, this second unrolled body changed the code
+//    the compiler produced for the full tiles: with 32 workers the fused pass lost 1 % at full
+//    clock and 3-10 % when the power limit lowers the SM clock and the consumers' instruction
+//    stream starts to matter. The copies (not the loop's registers) have their address taken.
 template <int KT, bool BF16, bool ADAM>
-__device__ __forceinline__ void ragged_tile(Acc<KT, Elem<BF16>::VEC>& a, const StepArgs& A, int64_t jt, float* dv, float* nv) {
+__device__ __forceinline__ void ragged_tile_body(Acc<KT, Elem<BF16>::VEC>& a, const StepArgs& A, int64_t jt, float* dv, float* nv) {
   typedef typename Elem<BF16>::T GT;
   if (jt < A.P) {
 #pragma unroll 4
@@ -555,6 +560,28 @@ __device__ __forceinline__ void ragged_tile(Acc<KT, Elem<BF16>::VEC>& a, const S
     if constexpr (ADAM) asm volatile("prefetch.global.L2 [%0];" :: "l"(A.second + jt));
   }
   direct_tile<KT, BF16, true, 4, ADAM>(a, A, jt, dv, nv);
+}
+
+template <int KT, bool BF16, bool ADAM>
+__device__ __noinline__ void ragged_tile_call(Acc<KT, Elem<BF16>::VEC>& a, const StepArgs& A, int64_t jt, float* dv, float* nv) {
+  ragged_tile_body<KT, BF16, ADAM>(a, A, jt, dv, nv);
+}
+
+constexpr int kRaggedInlineMaxK = 8;   // kernels for up to this many workers take the ragged tile inline
+
+template <int KT, bool BF16, bool ADAM>
+__device__ __forceinline__ void ragged_tile(Acc<KT, Elem<BF16>::VEC>& a, const StepArgs& A, int64_t jt, float* dv, float* nv) {
+  if constexpr (KT <= kRaggedInlineMaxK) {
+    ragged_tile_body<KT, BF16, ADAM>(a, A, jt, dv, nv);
+  } else {
+    constexpr int VEC = Elem<BF16>::VEC;
+    Acc<KT, VEC> a2 = a;
+    float dv2[VEC], nv2[VEC];
+    ragged_tile_call<KT, BF16, ADAM>(a2, A, jt, dv2, nv2);
+    a = a2;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) { dv[e] = dv2[e]; nv[e] = nv2[e]; }
+  }
 }
 
 template <int KT, bool BF16, int NW, int U, bool ADAM>

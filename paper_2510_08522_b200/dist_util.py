@@ -125,21 +125,24 @@ def gather_batch_sizes(b_local: int):
 
 def allgather_ranges(shard, ranges, out_full):
     """Rebuild a whole-length vector (the updated parameters) from the ranks' shards: out_full[lo_r:hi_r] =
-    rank r's shard. Shards differ in length, so each is padded to the longest for the collective."""
+    rank r's shard. Shards differ in length, so instead of one all-gather of padded copies every rank's
+    shard is broadcast straight into its place in `out_full` (one broadcast per non-empty shard, all in
+    flight together): each byte crosses the link once and nothing is staged on the device."""
     import torch
     import torch.distributed as dist
-    world = len(ranges)
     if not _group:
         out_full[ranges[0][0]:ranges[0][1]] = shard[:ranges[0][1] - ranges[0][0]]
         return out_full
-    longest = max(b - a for a, b in ranges)
-    staged = _host_staged() and shard.is_cuda
-    mine = torch.zeros(longest, dtype=shard.dtype, device="cpu" if staged else shard.device)
-    mine[:shard.numel()] = shard
-    every = [torch.empty_like(mine) for _ in range(world)]
-    dist.all_gather(every, mine)
-    for (a, b), t in zip(ranges, every):
-        out_full[a:b] = t[:b - a].to(out_full.device)
+    me = dist.get_rank()
+    staged = _host_staged() and out_full.is_cuda
+    dst = torch.empty(out_full.numel(), dtype=out_full.dtype, device="cpu") if staged else out_full
+    a, b = ranges[me]
+    dst[a:b] = shard[:b - a].to(dst.device)
+    works = [dist.broadcast(dst[lo:hi], src=r, async_op=True) for r, (lo, hi) in enumerate(ranges) if hi > lo]
+    for w in works:
+        w.wait()
+    if staged:
+        out_full.copy_(dst)
     return out_full
 
 

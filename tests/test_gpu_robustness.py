@@ -79,7 +79,7 @@ def test_destroyed_handles_are_refused():
                        out.data_ptr()) == Bn.ERR_HANDLE        # a handle of the other kind is not a step handle
 
 
-@pytest.mark.parametrize("idx,P", [(1, 300_007), (4, 2_000_003)])     # one launch per step / two launches per step
+@pytest.mark.parametrize("idx,P", [(1, 300_007), (4, 2_000_003)])
 def test_a_wait_that_runs_out_is_reported_and_cleared(idx, P):
     torch, D, Bn = _env()
     wl = W.WORKLOADS[idx].scaled(P=P, S=7)
@@ -100,8 +100,8 @@ def test_a_wait_that_runs_out_is_reported_and_cleared(idx, P):
         st2 = d.step(dp.grads, b, dp.params, dp.momentum, wl.lr, wl.beta, dp.prev_agg).cpu().numpy()
         assert not int(st2[Bn.ST_FLAGS]) & Bn.FLAG_INTERNAL
     per_poll_us = times[1 << 18] / (1 << 18) * 1e3
-    print("bounded wait: %s ms; %.3f us per poll -> 2^24 polls = %.2f s" % (times, per_poll_us, per_poll_us * (1 << 24) * 1e-6))
-    assert times[1 << 18] < 5000.0                               # the full budget (64 times this) stays well under minutes
+    print("bounded wait: %s ms; %.3f us per poll" % (times, per_poll_us))
+    assert times[1 << 18] < 5000.0                               # 2^18 polls is the fused pass's own budget: seconds, not minutes
     d.check_guards()
     d.close()
 
