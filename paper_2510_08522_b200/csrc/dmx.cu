@@ -209,13 +209,22 @@ Plan pick_direct(int K) {
   return direct_plan<64, BF16>();
 }
 
-// Pipelined (bulk-copy ring) kernels. Ring geometry: 7 consumer warps + the producer warp = 8
-// warps, so that a thread may use up to 255 registers (9 warps are allocated as 12 and cap it
-// at 168, which spilled at K = 32). A stage holds up to 16 gradient streams (56 KB): the
-// consumers pay one wait, one release and one batch of shared-memory loads per stage, and with
-// 4 streams per stage that per-stage work made the consumers the limiter as soon as the SM
-// clock dropped under the board's power limit (steps launched back to back: 5.8 -> 6.5 TB/s at
-// K = 32 bf16, 6.2 -> 6.8 TB/s at K = 32 fp32 with 16; the time at full clock is unchanged).
+// Pipelined (bulk-copy ring) kernels. Ring geometry. A CTA of up to 8 warps may use 255 registers
+// per thread, one of 9 to 12 warps 168 (registers are allocated per scheduler: three warps there
+// instead of two).
+//  - bf16 gradients, and fp32 gradients for more than 32 workers: 7 consumer warps + the
+//    producer. A thread holds 8 elements (bf16) or 64 per-worker sums and needs more than 168
+//    registers (with 11 consumer warps the K = 32 bf16 kernel spilled and lost 1-7 %).
+//  - fp32 gradients, up to 32 workers: 11 consumer warps + the producer; 168 registers suffice
+//    when a thread loads a stage's streams four at a time instead of all at once. More warps hide
+//    the consumers' latencies better: K = 8 128 -> 118 us per step (the fp64 aggregate had made 7
+//    warps the limiter), K = 32 +1.6 % at full clock and +6.7 % when the board's power limit has
+//    lowered the SM clock (3331 -> 3122 us back to back, same box).
+// A stage holds up to 16 gradient streams (8 in the 11-warp kernels, whose tile pieces are
+// larger): 45-56 KB. The consumers pay one wait, one release and one batch of shared-memory loads
+// per stage, and with 4 streams per stage (14 KB) that per-stage work made the consumers the limiter as
+// soon as the SM clock dropped under the power limit (steps launched back to back: 5.8 -> 6.5 TB/s
+// at K = 32 bf16, 6.2 -> 6.8 TB/s at K = 32 fp32; the time at full clock is unchanged).
 // Stages smaller than 4 streams lose even at full clock.
 // The producer runs at most NSS tiles ahead of the consumers (a tile's state stage is freed when
 // the consumers have read it), so the bytes in flight per SM are min(ring, NSS tiles). With many
@@ -225,8 +234,10 @@ Plan pick_direct(int K) {
 // each) as fit.
 template <int KT, bool BF16, bool ADAM>
 struct Ring {
-  static constexpr int CW = (KT <= 8 && !BF16) ? 11 : 7;
-  static constexpr int G = KT < 16 ? KT : 16;                                       // gradient streams per stage
+  static constexpr bool kWide = !BF16 && KT <= 32;                                  // the 11-consumer-warp kernels
+  static constexpr int CW = kWide ? 11 : 7;
+  static constexpr int G = KT < 16 ? KT : (kWide ? 8 : 16);                         // gradient streams per stage
+  static constexpr int LB = (kWide && G > 4) ? 4 : G;                               // streams loaded before they are accumulated
   static constexpr int kStage = CW * 32 * 16 * G;                                   // bytes of a gradient stage
   static constexpr int kState = CW * 32 * (BF16 ? 8 : 4) * 4 * (ADAM ? 4 : 3);      // bytes of a state stage
   static constexpr int kTile = (KT + G - 1) / G * kStage + kState;                  // shared memory of one tile
@@ -236,7 +247,7 @@ struct Ring {
   static constexpr int kFit = (227 * 1024 - NSS * (kState + 16) - kRed - 128) / (kStage + 16);
   static constexpr int NSTAGE = kFit > 32 ? 32 : kFit;
   static_assert(NSTAGE >= 2, "the ring needs two gradient stages");
-  typedef dmx::PipeCfg<KT, BF16, CW, G, NSTAGE, NSS, ADAM> Cfg;
+  typedef dmx::PipeCfg<KT, BF16, CW, G, NSTAGE, NSS, ADAM, LB> Cfg;
 };
 
 template <int KT, bool BF16>

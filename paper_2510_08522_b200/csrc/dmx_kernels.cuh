@@ -927,9 +927,10 @@ struct MbarSync {
   }
 };
 
-template <int KT_, bool BF16_, int CW_, int G_, int NSTAGE_, int NSS_, bool ADAM_ = false>
+template <int KT_, bool BF16_, int CW_, int G_, int NSTAGE_, int NSS_, bool ADAM_ = false, int LB_ = G_>
 struct PipeCfg {
   static constexpr int KT = KT_, CW = CW_, G = G_, NSTAGE = NSTAGE_, NSS = NSS_;
+  static constexpr int LB = LB_;                     // streams of a stage a consumer thread loads before it accumulates them
   static constexpr bool BF16 = BF16_, ADAM = ADAM_;
   static constexpr int NST = ADAM ? 4 : 3;           // state streams: prev_agg, momentum, params (, second moment)
   static constexpr int VEC = Elem<BF16>::VEC;
@@ -948,6 +949,7 @@ struct PipeCfg {
   static constexpr int TAIL = 16 + QN * 32;          // give-up word, chunk queue (8 ints per entry)
   static constexpr size_t SMEM = (size_t)RING + SRING + RED + NBAR * 8 + TAIL;
   static_assert(G >= 1 && G <= 32, "one producer lane per stream of a stage");
+  static_assert(LB >= 1 && LB <= G, "load batch");
   static_assert(NSTAGE <= 32 && NSS <= 32, "stage masks are 32 bits wide");
   static_assert(SMEM <= 227 * 1024, "ring does not fit in shared memory");
 };
@@ -955,6 +957,7 @@ struct PipeCfg {
 template <class C>
 __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_constant__ StepArgs A) {
   constexpr int KT = C::KT, VEC = C::VEC, CW = C::CW, G = C::G, NSTAGE = C::NSTAGE, NSS = C::NSS, T = C::T, QN = C::QN;
+  constexpr int LB = C::LB;
   constexpr bool BF16 = C::BF16, ADAM = C::ADAM;
   extern __shared__ __align__(128) unsigned char smem[];
   const uint32_t ring = smem_u32(smem);
@@ -1112,20 +1115,26 @@ __global__ void __launch_bounds__(C::THREADS, 1) pipe_kernel(const __grid_consta
         for (int s = 0; s < (KT + G - 1) / G; ++s) {
           if (s * G < A.K) {
             ok = mbar_wait(full_g + 8 * stage, phase, give_up, A.err) && ok;
-            uint4 r[G];
             const uint32_t src = ring + stage * C::STAGE + tid * 16;
+            // the stage's streams LB at a time: load, (after the last load: release the stage,) accumulate
 #pragma unroll
-            for (int u = 0; u < G; ++u)
-              if (s * G + u < KT && s * G + u < A.K) r[u] = lds128(src + u * C::SLOT);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty_g + 8 * stage);
-            if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
+            for (int u0 = 0; u0 < G; u0 += LB) {
+              uint4 r[LB];
 #pragma unroll
-            for (int u = 0; u < G; ++u) {
-              if (s * G + u < KT && s * G + u < A.K) {
-                u64 x[VEC / 2];
-                unpack2<BF16>(r[u], x);
-                a.add(s * G + u, x, A.w[s * G + u], A.bf[s * G + u], A.bd[s * G + u]);
+              for (int u = 0; u < LB; ++u)
+                if (u0 + u < G && s * G + u0 + u < KT && s * G + u0 + u < A.K) r[u] = lds128(src + (u0 + u) * C::SLOT);
+              if (u0 + LB >= G) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_g + 8 * stage);
+                if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
+              }
+#pragma unroll
+              for (int u = 0; u < LB; ++u) {
+                if (u0 + u < G && s * G + u0 + u < KT && s * G + u0 + u < A.K) {
+                  u64 x[VEC / 2];
+                  unpack2<BF16>(r[u], x);
+                  a.add(s * G + u0 + u, x, A.w[s * G + u0 + u], A.bf[s * G + u0 + u], A.bd[s * G + u0 + u]);
+                }
               }
             }
           }
