@@ -124,9 +124,11 @@ def step_bytes(wl, optimizer):
 
 
 L2_FLUSH_BELOW = 4 << 30      # workloads streaming less than this per step get an L2 flush between steps
+B2B_MIN_BYTES = 512 << 20     # ... and those streaming at least this much (4 x L2) are also timed back to back
 
 
-def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profile=True, optimizer="sgd", sustained=True):
+def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profile=True, optimizer="sgd", sustained=True,
+                 back_to_back=0):
     """Time `steps` steps of workload `wl` on `device`. Returns a dict of local measurements.
     Workloads whose step streams only a few times the L2's size get a 512 MB write between the
     (untimed) input generation and the timed step, so that no step starts on a warm L2."""
@@ -233,6 +235,20 @@ def run_workload(wl, steps, warmup, device, e2e_steps, sample_clocks=True, profi
         tail = sorted(sus[-max(20, n_sus // 4):])
         res["sustained"] = {"fused_kernel_ms": tail[len(tail) // 2], "first_fused_kernel_ms": sus[0], "launches": n_sus,
                             "clocks": sus_clocks}
+    if back_to_back > 0:
+        # whole steps launched straight behind one another inside ONE pair of events (only for workloads
+        # whose step streams several times the L2's size, so that no step finds its inputs cached): what a
+        # step costs the device once the launch and event latency around an isolated step is out of the picture
+        b = dp.batch_sizes()
+        for _ in range(3):
+            one_step(b)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(back_to_back):
+            one_step(b)
+        e1.record()
+        torch.cuda.synchronize()
+        res["back_to_back_ms"] = e0.elapsed_time(e1) / back_to_back
     d.close()
     if sample_clocks and world_is_one():
         # what plain reads of the same gradient buffers stream at in this run (context for the roofline)
@@ -358,7 +374,10 @@ def main():
         events (so the two launches keep their dependent-launch overlap), then the fused kernel's
         own time from a second pass with them."""
         peak_x, _ = measured_peak()
-        r_plain = run_workload(wlx, nsteps, args.warmup, device, 0, sample_clocks=False, profile=False, optimizer=args.optimizer)
+        nbx = step_bytes(wlx, args.optimizer)
+        b2b = 100 if B2B_MIN_BYTES <= nbx < L2_FLUSH_BELOW else 0
+        r_plain = run_workload(wlx, nsteps, args.warmup, device, 0, sample_clocks=False, profile=False, optimizer=args.optimizer,
+                               back_to_back=b2b)
         del r_plain["problem"]
         torch.cuda.empty_cache()
         r_prof = run_workload(wlx, nsteps, args.warmup, device, 0, sample_clocks=False, profile=True, optimizer=args.optimizer)
@@ -366,11 +385,16 @@ def main():
         torch.cuda.empty_cache()
         msx = r_plain["total_ms"] / len(r_plain["times"])
         fx = sum(r_prof["fused_ms"]) / len(r_prof["fused_ms"])
-        nbx = step_bytes(wlx, args.optimizer)
-        return {"workload": wlx.name, "value": nbx / msx / 1e6, "unit": UNIT, "ms_per_step": msx,
-                "steps_per_s": 1e3 / msx, "bytes_per_step": nbx, "fused_kernel_ms": fx,
-                "roofline_frac": nbx / fx / 1e6 / peak_x,
-                "l2": "flushed between steps" if r_plain["l2_flushed"] else "inputs larger than L2"}
+        out = {"workload": wlx.name, "value": nbx / msx / 1e6, "unit": UNIT, "ms_per_step": msx,
+               "steps_per_s": 1e3 / msx, "bytes_per_step": nbx, "fused_kernel_ms": fx,
+               "roofline_frac": nbx / fx / 1e6 / peak_x,
+               "l2": "flushed between steps" if r_plain["l2_flushed"] else "inputs larger than L2"}
+        if "back_to_back_ms" in r_plain:
+            out["back_to_back"] = {"ms_per_step": r_plain["back_to_back_ms"], "value": nbx / r_plain["back_to_back_ms"] / 1e6,
+                                   "unit": UNIT, "steps": b2b,
+                                   "what": "whole steps launched back to back between one pair of events, no flush: "
+                                           "a step streams more than four times the L2's size"}
+        return out
 
     also = None
     if args.also >= 0 and args.also != args.workload and world == 1:
