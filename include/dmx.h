@@ -165,8 +165,8 @@ int dmx_step(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_s
  * with ghat_j = g_j / (sqrt(vhat_j) + eps), the aggregate in units of Adam's running scale:
  *   out_state[12] = mean_j ghat_j     out_state[13] = var_j ghat_j (population variance over
  *   the P parameters)                 out_state[14] = sqrt(max(out_state[13], 0))
- * (dmx_step leaves 12..15 at 0.) This reading of "normalized variance / standard deviation
- * of gradients" under an adaptive optimizer is this library's: the paper gives no formula.
+ * (dmx_step leaves 12..15 at 0.) This reading of the gradient variance and standard deviation
+ * normalized for an adaptive optimizer is this library's: the paper gives no formula.
  */
 int dmx_step_adam(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes,
                   float* params, float* first_moment, float* second_moment, float lr, float beta1,

@@ -19,7 +19,7 @@ k training iterations of a cycle):
      with x_i the batch size used during the cycle.
 
 The paper fixes the action set, the clamp and the reward formula; it gives neither the layout
-of the state vector nor the policy network. Those are this build's definitions ("parity
+of the state vector nor the policy network. Those are this library's definitions ("parity
 unpinned" with respect to the paper): the state layout below, and a two-hidden-layer tanh MLP
 whose weights the caller supplies. Pinned by tests/test_ctl.py: hand-computed rewards and
 clamps, the action table, the MLP against torch.nn layers in fp64, softmax sampling

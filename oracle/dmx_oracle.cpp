@@ -16,7 +16,7 @@
 //     m <- b1 m + (1-b1) g, v <- b2 v + (1-b2) g^2, theta <- theta - lr mhat/(sqrt(vhat)+eps)
 //     with mhat = m/(1-b1^t), vhat = v/(1-b2^t). In Adam mode the state vector also carries
 //     mean, variance and standard deviation over the parameters of g_j/(sqrt(vhat_j)+eps),
-//     this build's reading of the "normalized" gradient statistics under an adaptive optimizer.
+//     this library's reading of the gradient statistics normalized for an adaptive optimizer.
 //   Section "State representation", "Training Statistical Efficiency Metrics": gradient
 //     statistics, sigma_norm and sigma^2_norm; Section "RL Agent Inference Evaluation",
 //     "Batch Size Adaptation Dynamics": the gradient noise scale.

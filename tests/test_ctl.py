@@ -2,7 +2,7 @@
 
 The paper fixes the action set {-100,-25,0,+25,+100}, the clamp to [32, 1024] and the reward
 formula (Sections "Action space and batch size adjustment" and "Reward function design"); those
-are pinned by hand-computed values. The policy network and the state layout are this build's
+are pinned by hand-computed values. The policy network and the state layout are this library's
 definitions; the network is pinned against torch.nn layers, the layout by one-hot probes.
 """
 import numpy as np
