@@ -315,7 +315,11 @@ int dmx_plan_chunks(int64_t P, int K, int grad_dtype, int tile_elems, int reside
  *                    state_len + i), and the window restarts; entry DMX_ST_FLAGS gets the OR of
  *                    the k flag words and spread 0. Other pushes leave window_out untouched.
  *                    *emitted (HOST, may be NULL) is set to 1 on the pushes that write, else 0.
- *                    Asynchronous, no allocation.
+ *                    Asynchronous, no allocation. The position inside the window is counted on the
+ *                    host, by call (which is why *emitted is known when the call returns, without
+ *                    waiting for the device): a handle's pushes must be issued one after the other
+ *                    (not concurrently from several threads), in the order of the steps, and on
+ *                    one stream, so that the device executes them in that same order.
  * Errors: DMX_ERR_ARG, DMX_ERR_NOMEM, DMX_ERR_HANDLE, DMX_ERR_CUDA.
  */
 typedef struct dmx_agg dmx_agg;
