@@ -246,6 +246,9 @@ int dmx_step_host(dmx_handle* h, const void* const* host_grad_ptrs, void* const*
  * between the two kernels and after finalize. dmx_get_profile waits for the last step's
  * events and returns the two durations in milliseconds. Errors: DMX_ERR_HANDLE,
  * DMX_ERR_ARG (no step recorded, or profiling off), DMX_ERR_CUDA.
+ * For timeline tools every step is also bracketed by NVTX ranges on the host ("dmx_step" or
+ * "dmx_step_adam", with "dmx fused pass" and "dmx finalize" inside); they cost a pointer test
+ * when no tool is attached.
  */
 int dmx_set_profiling(dmx_handle* h, int on);
 int dmx_get_profile(dmx_handle* h, float* fused_ms, float* finalize_ms);

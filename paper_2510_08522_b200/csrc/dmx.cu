@@ -11,6 +11,8 @@
 #include <unordered_map>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "dmx_host.h"
 #include "dmx_kernels.cuh"
 
@@ -522,6 +524,15 @@ namespace {
 
 struct AdamParams { float* second; float beta2, eps; int64_t t; };
 
+// A named range around the enqueueing of a step's launches, for timeline tools (NVTX; a call costs
+// a pointer test when no tool is attached).
+struct TraceRange {
+  explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+  ~TraceRange() { nvtxRangePop(); }
+  TraceRange(const TraceRange&) = delete;
+  TraceRange& operator=(const TraceRange&) = delete;
+};
+
 // One step with either update; `ap` is null for SGD with momentum.
 int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_sizes, float* params,
               float* momentum, float lr, float beta, float* prev_agg, float* out_state, void* cuda_stream,
@@ -580,11 +591,16 @@ int step_impl(dmx_handle* h, const void* const* grad_ptrs, const int32_t* batch_
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const bool prof = h->profiling;
+  const TraceRange step_range(ap ? "dmx_step_adam" : "dmx_step");
   if (prof && !cuda_ok(cudaEventRecord(h->ev[0], stream))) return DMX_ERR_CUDA;
-  if (ap) h->plan.kernel_adam<<<h->plan.grid, h->plan.threads, h->plan.smem_adam, stream>>>(A);
-  else h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A);
+  {
+    const TraceRange r("dmx fused pass");
+    if (ap) h->plan.kernel_adam<<<h->plan.grid, h->plan.threads, h->plan.smem_adam, stream>>>(A);
+    else h->plan.kernel<<<h->plan.grid, h->plan.threads, h->plan.smem, stream>>>(A);
+  }
   if (!cuda_ok(cudaGetLastError())) return DMX_ERR_CUDA;
   if (prof && !cuda_ok(cudaEventRecord(h->ev[1], stream))) return DMX_ERR_CUDA;
+  const TraceRange fin_range("dmx finalize");
   // one block per chunk-row column, one warp per segment unit. Launched as a programmatic
   // dependent of the fused pass: its blocks may become resident while that kernel drains and
   // wait (griddepcontrol.wait) for its completion, which hides the launch latency between the
