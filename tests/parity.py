@@ -206,6 +206,40 @@ def cond_vectors_t(torch, grads, b, params_in, momentum_in, lr, beta):
     return cg, cm, ct
 
 
+def cond_vectors_adam_t(torch, grads, b, params_in, m_in, v_in, lr, beta1, beta2, eps, t):
+    """cond_vectors_adam (without the update's own scales) on torch tensors: gradients as stored
+    (fp32 or bf16 tensors, widened exactly), state as fp32 tensors; float64 tensors on their device."""
+    w = np.asarray(b, np.float64) / float(np.sum(b))
+    n, dev = grads[0].numel(), grads[0].device
+    cg = torch.zeros(n, dtype=torch.float64, device=dev)
+    g = torch.zeros(n, dtype=torch.float64, device=dev)
+    for k, x in enumerate(grads):
+        x64 = x.to(torch.float64)
+        g.add_(x64, alpha=float(w[k]))
+        cg.add_(x64.abs_(), alpha=float(w[k]))
+    b1, b2 = float(np.float32(beta1)), float(np.float32(beta2))
+    m64, v64 = m_in.to(torch.float64), v_in.to(torch.float64)
+    cm = (b1 * m64).abs_() + (1 - b1) * cg
+    cv = b2 * v64.abs() + (1 - b2) * 2 * cg * cg
+    c1, c2 = 1 / (1 - b1 ** t), 1 / (1 - b2 ** t)
+    m_new = b1 * m64 + (1 - b1) * g
+    v_new = b2 * v64 + (1 - b2) * g * g
+    root = torch.sqrt(v_new * c2)
+    den = root + float(np.float32(eps))
+    tiny = torch.full_like(den, 1e-300)
+    u = m_new * c1 / torch.maximum(den, tiny)
+    cu = c1 * cm / torch.maximum(den, tiny) + u.abs() * c2 * cv / torch.maximum(2 * root * den, tiny)
+    ct = params_in.to(torch.float64).abs_() + abs(float(np.float32(lr))) * (u.abs() + cu)
+    return cg, cm, cv, ct
+
+
+def seg_scales_range_t(torch, cg, seg, lo):
+    """seg_scales with an offset on a torch tensor: the elements [lo, lo + len(cg)) of the problem."""
+    cs = torch.cat([torch.zeros(1, dtype=torch.float64, device=cg.device), torch.cumsum(cg * cg, 0)])
+    idx = torch.as_tensor(np.clip(np.asarray(seg, np.int64) - lo, 0, cg.numel()), device=cg.device)
+    return (cs[idx[1:]] - cs[idx[:-1]]).cpu().numpy()
+
+
 def vec_err_t(torch, gpu, ref, cond):
     """vec_err on torch tensors (fp32 values, float64 scale)."""
     ref64 = ref.to(torch.float64)

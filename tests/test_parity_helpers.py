@@ -25,6 +25,19 @@ def test_torch_scales_equal_numpy_scales():
     assert np.allclose(PT.seg_scales(ref[0], seg), PT.seg_scales_t(torch, got[0], seg), rtol=1e-10)
 
 
+def test_torch_adam_scales_equal_numpy_scales():
+    grads, b, params, mom = _problem(seed=6)
+    v = np.abs(_problem(seed=7)[2]) * 1e-2
+    ref = PT.cond_vectors_adam(grads, b, params, mom, v, 1e-3, 0.9, 0.999, 1e-8, 5)
+    got = PT.cond_vectors_adam_t(torch, [torch.from_numpy(g) for g in grads], b, torch.from_numpy(params), torch.from_numpy(mom),
+                                 torch.from_numpy(v), 1e-3, 0.9, 0.999, 1e-8, 5)
+    for a, t in zip(ref, got):
+        assert np.allclose(a, t.numpy(), rtol=1e-12, atol=0)
+    seg = [0, 1, 1, 7, 4000, 4099]
+    for lo, hi in ((0, 4099), (5, 3000), (3999, 4099)):
+        assert np.allclose(PT.seg_scales(ref[0][lo:hi], seg, lo), PT.seg_scales_range_t(torch, got[0][lo:hi], seg, lo), rtol=1e-10)
+
+
 def test_torch_scales_widen_bf16_exactly():
     grads, b, params, mom = _problem(seed=4)
     gb = [torch.from_numpy(g).to(torch.bfloat16) for g in grads]
